@@ -1,0 +1,171 @@
+"""Pins for the oracle's packed-segment statistics and the Delta-IFD rule
+(Eq. 3, Eq. 4, three-zone rule): unpacked per-sequence runs, a hand-worked
+table, invariances and edge cases.  CPU only."""
+
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import npd_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "delta_ifd_table.txt")
+
+
+def _packed(seed=0):
+    rng = np.random.default_rng(seed)
+    lens = [5, 1, 9, 3, 7]
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    T, d, V = int(cu[-1]), 4, 10
+    H = rng.standard_normal((T, d))
+    W = rng.standard_normal((V, d))
+    Zt = rng.standard_normal((T, V)) * 2
+    y = rng.integers(0, V, size=T)
+    m = (rng.random(T) < 0.6).astype(np.uint8)
+    for s in range(len(lens)):
+        y[cu[s + 1] - 1] = -100
+        m[cu[s + 1] - 1] = 0
+    y[2] = -100            # an ignored label on a token that still carries KL
+    m[2] = 1
+    return cu, H, W, Zt, y, m
+
+
+def test_segment_sums_equal_unpacked_per_sequence_runs():
+    cu, H, W, Zt, y, m = _packed()
+    kl, ns, nt = orc.kd_token_losses(H, W, Zt, y, m, 1.5)
+    kl_sum, s_sum, t_sum, cnt = orc.segment_stats(cu, m, y, kl, ns, nt)
+    for s in range(len(cu) - 1):
+        sl = slice(cu[s], cu[s + 1])
+        k1, s1, t1 = orc.kd_token_losses(H[sl], W, Zt[sl], y[sl], m[sl], 1.5)
+        assert math.isclose(kl_sum[s], k1.sum(), rel_tol=1e-13, abs_tol=1e-15)
+        assert math.isclose(s_sum[s], s1.sum(), rel_tol=1e-13, abs_tol=1e-15)
+        assert math.isclose(t_sum[s], t1.sum(), rel_tol=1e-13, abs_tol=1e-15)
+        assert cnt[s] == int(((m[sl] == 1) & (y[sl] >= 0)).sum())
+    assert cnt.dtype == np.int32
+    assert cnt.sum() == int(((m == 1) & (y >= 0)).sum())
+    assert math.isclose(kl_sum.sum(), kl.sum(), rel_tol=1e-13)
+
+
+def test_count_excludes_ignored_labels_but_kl_sum_does_not():
+    cu, H, W, Zt, y, m = _packed()
+    kl, ns, nt = orc.kd_token_losses(H, W, Zt, y, m, 1.0)
+    kl_sum, _, _, cnt = orc.segment_stats(cu, m, y, kl, ns, nt)
+    seg0 = slice(cu[0], cu[1])
+    assert cnt[0] == int(((m[seg0] == 1) & (y[seg0] >= 0)).sum())
+    assert kl[2] > 0 and ns[2] == 0          # token 2: KL but no label
+    assert kl_sum[0] >= kl[2]
+
+
+def test_permuting_segments_permutes_statistics():
+    cu, H, W, Zt, y, m = _packed(3)
+    kl, ns, nt = orc.kd_token_losses(H, W, Zt, y, m, 1.0)
+    base = orc.segment_stats(cu, m, y, kl, ns, nt)
+    perm = [3, 0, 4, 2, 1]
+    idx = np.concatenate([np.arange(cu[s], cu[s + 1]) for s in perm])
+    cu_p = np.concatenate([[0], np.cumsum([cu[s + 1] - cu[s] for s in perm])])
+    got = orc.segment_stats(cu_p, m[idx], y[idx], kl[idx], ns[idx], nt[idx])
+    for a, b in zip(base, got):
+        assert np.allclose(np.asarray(a)[perm], b, rtol=1e-14)
+
+
+def test_segment_ids_and_validation():
+    cu = np.array([0, 2, 3, 7], dtype=np.int32)
+    assert orc.segment_ids(cu, 7).tolist() == [0, 0, 1, 2, 2, 2, 2]
+    assert orc.segment_ids(cu, 7).dtype == np.int32
+    assert orc.validate_cu_seqlens(cu, 7)
+    assert not orc.validate_cu_seqlens(cu, 8)                  # does not end at T
+    assert not orc.validate_cu_seqlens([1, 2, 7], 7)           # does not start at 0
+    assert not orc.validate_cu_seqlens([0, 3, 3, 7], 7)        # empty segment
+    assert not orc.validate_cu_seqlens([0, 5, 4, 7], 7)        # not increasing
+    assert not orc.validate_cu_seqlens([0], 0)
+
+
+def _read_golden():
+    rows = []
+    with open(GOLDEN) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            left, right = line.split("|")
+            l, r = left.split(), right.split()
+            rows.append(dict(cc=int(l[1]), cu=int(l[2]), tc=float(l[3]), tu=float(l[4]),
+                             sc=float(l[5]), su=float(l[6]), ifd_t=float(r[0]), ifd_s=float(r[1]),
+                             delta=float(r[2]), keep=int(r[3]), keep2=int(r[4])))
+    return rows
+
+
+@pytest.mark.parametrize("dtype", [np.float64, np.float32])
+def test_hand_worked_table(dtype):
+    rows = _read_golden()
+    n = len(rows)
+    count = np.zeros(2 * n, dtype=np.int32)
+    t_sum = np.zeros(2 * n)
+    s_sum = np.zeros(2 * n)
+    for i, r in enumerate(rows):
+        count[2 * i], count[2 * i + 1] = r["cc"], r["cu"]
+        t_sum[2 * i], t_sum[2 * i + 1] = r["tc"], r["tu"]
+        s_sum[2 * i], s_sum[2 * i + 1] = r["sc"], r["su"]
+    cond = np.arange(n) * 2
+    unc = cond + 1
+    it, is_, dl, keep, nk = orc.delta_ifd_select(cond, unc, s_sum, t_sum, count, 0.0, 1.0,
+                                                 dtype=dtype)
+    assert it.dtype == dtype and dl.dtype == dtype and keep.dtype == np.uint8
+    for i, r in enumerate(rows):
+        for got, want in ((it[i], r["ifd_t"]), (is_[i], r["ifd_s"]), (dl[i], r["delta"])):
+            assert (math.isnan(got) and math.isnan(want)) or got == want
+        assert keep[i] == r["keep"]
+    assert nk == sum(r["keep"] for r in rows)
+    _, _, _, keep2, nk2 = orc.delta_ifd_select(cond, unc, s_sum, t_sum, count, 0.0, 1.0,
+                                               require_teacher_ifd_le_1=True, dtype=dtype)
+    assert keep2.tolist() == [r["keep2"] for r in rows]
+    assert nk2 == sum(r["keep2"] for r in rows)
+
+
+def test_teacher_equal_to_student_is_kept_and_scaling_leaves_delta_unchanged():
+    rng = np.random.default_rng(0)
+    n = 8
+    count = rng.integers(1, 20, size=2 * n).astype(np.int32)
+    s_sum = rng.random(2 * n) * 10 + 0.1
+    cond, unc = np.arange(n) * 2, np.arange(n) * 2 + 1
+    _, _, dl, keep, nk = orc.delta_ifd_select(cond, unc, s_sum, s_sum, count, 0.0, 0.8)
+    assert np.all(dl == 0) and np.all(keep == 1) and nk == n
+    t_sum = rng.random(2 * n) * 10 + 0.1
+    base = orc.delta_ifd_select(cond, unc, s_sum, t_sum, count, 0.0, 0.8)
+    scale = np.repeat(rng.random(n) * 5 + 0.5, 2)       # one constant per sample
+    scaled = orc.delta_ifd_select(cond, unc, s_sum * scale, t_sum * scale, count, 0.0, 0.8)
+    assert np.allclose(base[2], scaled[2], rtol=1e-12)
+    assert np.array_equal(base[3], scaled[3])
+
+
+def test_ifd_is_ratio_of_token_means_not_sums():
+    # cond: 4 tokens summing to 8 (mean 2); uncond: 2 tokens summing to 8 (mean 4)
+    ifd = orc.ifd_scores([0], [1], [8.0, 8.0], [4, 2])
+    assert ifd[0] == 0.5
+
+
+def test_pair_maps_are_arbitrary_indices():
+    count = np.array([2, 4, 1, 8], dtype=np.int32)
+    s = np.array([2.0, 4.0, 3.0, 8.0])
+    t = np.array([4.0, 4.0, 1.0, 4.0])
+    it, is_, dl, keep, nk = orc.delta_ifd_select([3, 0], [2, 1], s, t, count, 0.0, 1.0)
+    # sample 0: cond=3, unc=2 -> T: (4/8)/(1/1)=0.5 ; S: (8/8)/(3/1)=1/3
+    assert it[0] == 0.5 and math.isclose(is_[0], 1 / 3)
+    # sample 1: cond=0, unc=1 -> T: (4/2)/(4/4)=2 ; S: (2/2)/(4/4)=1
+    assert it[1] == 2.0 and is_[1] == 1.0 and dl[1] == 1.0 and keep[1] == 1
+    assert nk == 2
+
+
+def test_zero_denominator_and_empty_are_rejected():
+    count = np.array([3, 3, 0, 2], dtype=np.int32)
+    z = np.array([1.0, 0.0, 0.0, 1.0])
+    it, is_, dl, keep, nk = orc.delta_ifd_select([0, 2], [1, 3], z, z, count, -10, 10)
+    assert np.all(np.isnan(dl)) and keep.tolist() == [0, 0] and nk == 0
+
+
+def test_nearest_rank_percentile():
+    assert orc.nearest_rank_percentile([5, 1, 3, 2, 4], 0.8) == 4
+    assert orc.nearest_rank_percentile([5, 1, 3, 2, 4], 0.81) == 5
+    assert orc.nearest_rank_percentile([1, float("nan"), 2, 3, 4, 5], 0.2) == 1
+    assert orc.nearest_rank_percentile(np.arange(1, 11), 0.8) == 8
