@@ -1,0 +1,207 @@
+/*
+ * npd.h - C ABI of the packed-sequence distillation loss step of Near-Policy
+ * Distillation (NPD), implemented as hand-written CUDA kernels for NVIDIA B200
+ * (sm_100a).
+ *
+ * What the library computes (paper notation; T packed tokens, d hidden size,
+ * V vocabulary, S packed segments, tau softmax temperature):
+ *
+ *   O_S = H W^T                         Algorithm 1, "Compute Student Logits"
+ *                                       (LM head only; the transformer body is
+ *                                       the caller's)
+ *   p_T = Softmax(O_T / tau),           Algorithm 1, "Compute Probs"
+ *   p_S = Softmax(O_S / tau)
+ *   kl[t]  = m_t * sum_c p_T(c) log(p_T(c)/p_S(c))          Eq. 2, with the
+ *            support taken as the whole vocabulary (dense teacher logits; an
+ *            entry of -inf removes a class from the support)
+ *   nll_student[t] = -m_t [y_t>=0] log Softmax(O_S[t])[y_t]   cross-entropy
+ *   nll_teacher[t] = -m_t [y_t>=0] log Softmax(O_T[t])[y_t]   behind Eq. 3
+ *   dO_S[t,c] = grad_scale * m_t * (p_S(c) - p_T(c)) / tau    gradient of Eq. 2
+ *   dH = dO_S W,   dW = dO_S^T H                              Algorithm 1, "Update"
+ *   per-segment sums and counts over cu_seqlens               inputs of Eq. 3
+ *   IFD = L(A|Q)/L(A) (Eq. 3), Delta = IFD_T - IFD_S (Eq. 4),
+ *   keep = lo <= Delta <= hi (Proximal Learning Zone, Section 3.2)
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless the comment says HOST.
+ *   - The caller owns every buffer.  The library allocates no device memory,
+ *     keeps no problem state between calls and only enqueues work on the given stream
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *     Results are ready when the stream has been synchronised.
+ *   - Return value: NPD_OK (0) or a negative npd_status.  Argument errors are
+ *     found on the host before anything is launched.  Errors found on the device
+ *     (malformed cu_seqlens, a bounded wait that ran out) are recorded in the
+ *     workspace and read with npd_last_status().
+ *   - No exceptions, no abort(), no device traps.  Device-side waits are bounded.
+ *   - Needs a device of compute capability 10.x; otherwise NPD_EARCH.
+ */
+#ifndef NPD_H_
+#define NPD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum npd_status {
+  NPD_OK = 0,
+  NPD_EINVAL = -1,      /* null pointer, bad size field, non-positive dimension, tau <= 0 */
+  NPD_ESHAPE = -2,      /* d not a multiple of 64, a row stride smaller than the row, S > T */
+  NPD_EALIGN = -3,      /* a base pointer or row stride of a tensor operand not 16-byte aligned */
+  NPD_ESEQ = -4,        /* cu_seqlens malformed (found on the device) */
+  NPD_EARCH = -5,       /* current device is not compute capability 10.x */
+  NPD_EWORKSPACE = -6,  /* workspace NULL, misaligned or smaller than npd_workspace_bytes() */
+  NPD_ECUDA = -7,       /* a CUDA runtime or driver call failed */
+  NPD_ETIMEOUT = -8,    /* a bounded device-side wait expired (found on the device) */
+  NPD_EUNSUPPORTED = -9 /* a documented option that this build does not implement */
+} npd_status;
+
+enum { NPD_DTYPE_BF16 = 0, NPD_DTYPE_F32 = 1 };
+
+/* flags of npd_kd_args */
+enum {
+  NPD_KD_ACCUMULATE_DW = 1  /* add into d_weight instead of overwriting it (f32 d_weight only) */
+};
+
+/*
+ * Arguments of the fused KD forward+backward (Algorithm 1, Phase 3, lines
+ * "Compute Student Logits" to "Update", restricted to the LM head and Eq. 2).
+ *
+ * Layouts are row-major with explicit row strides in ELEMENTS.  hidden, weight,
+ * teacher, d_hidden and d_weight must be 16-byte aligned with row strides that
+ * are multiples of 16 bytes (8 bf16 elements).  d must be a multiple of 64.
+ * Any T >= 1, V >= 1 is accepted (ragged tiles are masked in the kernels).
+ */
+typedef struct npd_kd_args {
+  size_t size;               /* = sizeof(npd_kd_args); checked */
+  int32_t T, d, V, S;
+  const void* hidden;        /* bf16 [T, ldh]   H                                  */
+  const void* weight;        /* bf16 [V, ldw]   W (LM head, no bias)               */
+  const void* teacher;       /* bf16 [T, ldt]   O_T, ldt >= V; columns >= V ignored */
+  int64_t ldh, ldw, ldt;
+  int32_t teacher_dtype;     /* NPD_DTYPE_BF16 (NPD_DTYPE_F32: NPD_EUNSUPPORTED)    */
+  int32_t reserved0;
+  const int32_t* cu_seqlens; /* [S+1] cu[0]=0, strictly increasing, cu[S]=T; may be NULL
+                                (then S is ignored and nothing is validated)       */
+  const uint8_t* loss_mask;  /* [T] 1 = token carries loss; NULL = all ones         */
+  const int32_t* labels;     /* [T] class the position must predict, <0 = none;
+                                NULL = no NLL outputs                              */
+  float temperature;         /* tau > 0                                             */
+  float grad_scale;          /* dL/d(sum_t kl[t]); e.g. 1/n_loss                    */
+  /* outputs (each may be NULL unless noted) */
+  float* kl;                 /* [T] required                                        */
+  float* nll_student;        /* [T]                                                 */
+  float* nll_teacher;        /* [T]                                                 */
+  void* d_hidden;            /* bf16 [T, ldh]; NULL (with d_weight NULL) = forward only */
+  void* d_weight;            /* bf16 or f32 [V, ldw]; both gradients or neither     */
+  int32_t d_weight_dtype;    /* NPD_DTYPE_BF16 or NPD_DTYPE_F32                     */
+  int32_t flags;
+  int32_t grad_chunk_cols;   /* vocabulary columns of logit-gradient tiles that may be in
+                                flight between the gradient kernel and the two
+                                contractions; 0 = library default.  Bounds the scratch. */
+  int32_t reserved1;
+  void* workspace;           /* >= npd_workspace_bytes(), 1024-byte aligned         */
+  size_t workspace_bytes;
+} npd_kd_args;
+
+/* HOST.  Bytes of workspace npd_kd_fwd_bwd needs for these arguments (pointers
+ * inside args are not read).  Depends on T, d, V, grad_chunk_cols, on whether
+ * gradients are requested and on the device's SM count. */
+int npd_workspace_bytes(const npd_kd_args* args, size_t* out_bytes);
+
+/* Fused forward + backward of the distillation term (see the struct).  `args`
+ * is a HOST struct holding device pointers.  Enqueues on `cuda_stream`. */
+int npd_kd_fwd_bwd(const npd_kd_args* args, void* cuda_stream);
+
+/*
+ * Same computation from HOST buffers, for callers whose step inputs arrive in
+ * host memory.  `host` and `dev` describe the same problem: `dev` is a complete,
+ * valid npd_kd_args of device buffers (used as staging), `host` holds HOST
+ * pointers for the per-step inputs (hidden, teacher, cu_seqlens, loss_mask,
+ * labels; pinned memory for overlap) and for the per-token outputs (kl,
+ * nll_student, nll_teacher).  The weight is a resident parameter and the two
+ * gradients stay on the device: host->weight, d_hidden, d_weight are ignored.
+ * The call copies the inputs in, runs npd_kd_fwd_bwd(dev) and copies the
+ * per-token outputs back, all asynchronously on `cuda_stream`.
+ */
+int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* cuda_stream);
+
+/*
+ * Per-sample statistics for the Delta-IFD filter (the sums behind Eq. 3):
+ *   kl_sum[s]    = sum_{t in s} m_t kl[t]
+ *   nll_s_sum[s] = sum_{t in s} m_t [y_t>=0] nll_student[t]     (same for teacher)
+ *   count[s]     = sum_{t in s} m_t [y_t>=0]                    (bit-exact)
+ *   seg_id[t]    = s with cu[s] <= t < cu[s+1]                  (optional)
+ * Sums are taken in fp32 in a fixed order (deterministic).  kl / nll_* / the
+ * three sum outputs may be NULL in matching pairs.  loss_mask NULL = all ones,
+ * labels NULL = every label valid.  `status` (int32[1], may be NULL) receives
+ * NPD_ESEQ if cu_seqlens is malformed, else is left untouched.
+ */
+int npd_segment_stats(int32_t T, int32_t S, const int32_t* cu_seqlens,
+                      const uint8_t* loss_mask, const int32_t* labels,
+                      const float* kl, const float* nll_student, const float* nll_teacher,
+                      float* kl_sum, float* nll_s_sum, float* nll_t_sum,
+                      int32_t* count, int32_t* seg_id, int32_t* status, void* cuda_stream);
+
+/* flags of npd_select */
+enum {
+  NPD_SELECT_TEACHER_IFD_LE_1 = 1 /* also require IFD_Teacher <= 1 (Section 3.2, zone text) */
+};
+
+/*
+ * Delta-IFD score and selection (Eq. 3, Eq. 4, three-zone rule of Section 3.2).
+ * Sample i is described by two segments: cond_seg[i] holds prompt+answer with the
+ * prompt masked (L(A|Q)), uncond_seg[i] the answer alone (L(A)).  With
+ * L = nll_sum / count (token mean), in fp32 with IEEE division:
+ *   ifd_X[i] = L_X(cond) / L_X(uncond),  X in {teacher, student}
+ *   delta[i] = ifd_teacher[i] - ifd_student[i]
+ *   keep[i]  = lo <= delta[i] <= hi   (both inclusive; NaN never kept)
+ * A sample with an empty segment (count 0) or a zero denominator scores NaN.
+ * n_keep[0] = number of kept samples.  ifd_* and delta may be NULL.
+ */
+int npd_select(int32_t N, const int32_t* cond_seg, const int32_t* uncond_seg,
+               const float* nll_s_sum, const float* nll_t_sum, const int32_t* count,
+               int32_t S, float lo, float hi, int32_t flags,
+               float* ifd_teacher, float* ifd_student, float* delta,
+               uint8_t* keep, int32_t* n_keep, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, then reads the device-side status word of a
+ * workspace that npd_kd_fwd_bwd used into *host_status (HOST): NPD_OK,
+ * NPD_ESEQ or NPD_ETIMEOUT.  Returns NPD_ECUDA if the stream itself failed. */
+int npd_last_status(const void* workspace, void* cuda_stream, int32_t* host_status);
+
+/* HOST.  Static description of a status code. */
+const char* npd_strerror(int status);
+
+/* HOST.  Number of kernel launches the last npd_kd_fwd_bwd call on this thread
+ * enqueued (for launch accounting in benchmarks). */
+int npd_last_launch_count(void);
+
+/* out_mode of npd_gemm_bf16 */
+enum {
+  NPD_GEMM_STORE_F32 = 0,  /* D = acc                       */
+  NPD_GEMM_ADD_F32 = 1,    /* D += acc (one owner per tile) */
+  NPD_GEMM_STORE_BF16 = 2, /* D = bf16(acc)                 */
+  NPD_GEMM_ATOMIC_F32 = 3, /* D += acc with atomics (split-K; D must be initialised) */
+  NPD_GEMM_ADD_BF16 = 4    /* D = bf16(D + acc)             */
+};
+
+/*
+ * The tensor-core contraction behind the two backward products (dH = dO_S W and
+ * dW = dO_S^T H, the chain rule through Algorithm 1's student-logit step),
+ * exposed as a building block:
+ *     D[M,N] (+)= sum_k A[m,k] * B[n,k]      bf16 inputs, fp32 accumulation.
+ * An operand is K-major (memory [rows][K], x_mn_major = 0, ld >= K) or MN-major
+ * (memory [K][rows], x_mn_major = 1, ld >= rows).  Pointers 16-byte aligned, row
+ * strides multiples of 8 elements.  k_splits > 1 needs NPD_GEMM_ATOMIC_F32.
+ */
+int npd_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32_t a_mn_major,
+                  const void* B, int64_t ldb, int32_t b_mn_major, void* out, int64_t ldo,
+                  int32_t out_mode, int32_t k_splits, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NPD_H_ */

@@ -1,0 +1,231 @@
+"""ctypes binding of the C-ABI library (include/npd.h).
+
+Argument marshalling only: every step of the computation runs in the library's
+CUDA kernels.  PyTorch supplies device memory and streams.  There is no CPU or
+PyTorch fallback: if the library is not built the first call raises.
+"""
+
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnpd.so")
+
+NPD_OK = 0
+NPD_EINVAL, NPD_ESHAPE, NPD_EALIGN, NPD_ESEQ, NPD_EARCH = -1, -2, -3, -4, -5
+NPD_EWORKSPACE, NPD_ECUDA, NPD_ETIMEOUT, NPD_EUNSUPPORTED = -6, -7, -8, -9
+NPD_DTYPE_BF16, NPD_DTYPE_F32 = 0, 1
+NPD_KD_ACCUMULATE_DW = 1
+NPD_SELECT_TEACHER_IFD_LE_1 = 1
+NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32, NPD_GEMM_ADD_BF16 = range(5)
+
+EXPORTS = ("npd_workspace_bytes", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
+           "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16")
+
+
+class NpdError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+class npd_kd_args(C.Structure):
+    _fields_ = [
+        ("size", C.c_size_t),
+        ("T", C.c_int32), ("d", C.c_int32), ("V", C.c_int32), ("S", C.c_int32),
+        ("hidden", C.c_void_p), ("weight", C.c_void_p), ("teacher", C.c_void_p),
+        ("ldh", C.c_int64), ("ldw", C.c_int64), ("ldt", C.c_int64),
+        ("teacher_dtype", C.c_int32), ("reserved0", C.c_int32),
+        ("cu_seqlens", C.c_void_p), ("loss_mask", C.c_void_p), ("labels", C.c_void_p),
+        ("temperature", C.c_float), ("grad_scale", C.c_float),
+        ("kl", C.c_void_p), ("nll_student", C.c_void_p), ("nll_teacher", C.c_void_p),
+        ("d_hidden", C.c_void_p), ("d_weight", C.c_void_p),
+        ("d_weight_dtype", C.c_int32), ("flags", C.c_int32),
+        ("grad_chunk_cols", C.c_int32), ("reserved1", C.c_int32),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+    ]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded library.  Raises if it has not been built (no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2605_05940_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        l = C.CDLL(LIB_PATH)
+        l.npd_strerror.restype = C.c_char_p
+        l.npd_strerror.argtypes = [C.c_int]
+        l.npd_workspace_bytes.argtypes = [C.POINTER(npd_kd_args), C.POINTER(C.c_size_t)]
+        l.npd_kd_fwd_bwd.argtypes = [C.POINTER(npd_kd_args), C.c_void_p]
+        l.npd_kd_fwd_bwd_host.argtypes = [C.POINTER(npd_kd_args), C.POINTER(npd_kd_args), C.c_void_p]
+        l.npd_segment_stats.argtypes = [C.c_int32, C.c_int32] + [C.c_void_p] * 13
+        l.npd_select.argtypes = ([C.c_int32] + [C.c_void_p] * 5 + [C.c_int32, C.c_float, C.c_float, C.c_int32]
+                                 + [C.c_void_p] * 6)
+        l.npd_last_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
+        l.npd_last_launch_count.argtypes = []
+        l.npd_gemm_bf16.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int32,
+                                    C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64,
+                                    C.c_int32, C.c_int32, C.c_void_p]
+        _lib = l
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().npd_strerror(int(code)).decode()
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(rc: int, where: str):
+    if rc != NPD_OK:
+        raise NpdError(rc, where)
+
+
+def make_kd_args(hidden, weight, teacher, *, cu_seqlens=None, loss_mask=None, labels=None,
+                 temperature=1.0, grad_scale=1.0, kl=None, nll_student=None, nll_teacher=None,
+                 d_hidden=None, d_weight=None, flags=0, grad_chunk_cols=0,
+                 workspace=None) -> npd_kd_args:
+    """Fill an npd_kd_args from tensors (device tensors, or host tensors for the
+    `host` argument of npd_kd_fwd_bwd_host)."""
+    a = npd_kd_args()
+    a.size = C.sizeof(npd_kd_args)
+    a.T, a.d = hidden.shape
+    a.V = weight.shape[0]
+    a.S = 0 if cu_seqlens is None else cu_seqlens.numel() - 1
+    a.hidden, a.weight, a.teacher = _ptr(hidden), _ptr(weight), _ptr(teacher)
+    a.ldh, a.ldw, a.ldt = hidden.stride(0), weight.stride(0), teacher.stride(0)
+    a.teacher_dtype = NPD_DTYPE_F32 if teacher.dtype == torch.float32 else NPD_DTYPE_BF16
+    a.cu_seqlens, a.loss_mask, a.labels = _ptr(cu_seqlens), _ptr(loss_mask), _ptr(labels)
+    a.temperature, a.grad_scale = float(temperature), float(grad_scale)
+    a.kl, a.nll_student, a.nll_teacher = _ptr(kl), _ptr(nll_student), _ptr(nll_teacher)
+    a.d_hidden, a.d_weight = _ptr(d_hidden), _ptr(d_weight)
+    a.d_weight_dtype = (NPD_DTYPE_F32 if d_weight is not None and d_weight.dtype == torch.float32
+                        else NPD_DTYPE_BF16)
+    a.flags, a.grad_chunk_cols = int(flags), int(grad_chunk_cols)
+    if workspace is not None:
+        a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+    return a
+
+
+def npd_workspace_bytes(args: npd_kd_args) -> int:
+    out = C.c_size_t(0)
+    _check(lib().npd_workspace_bytes(C.byref(args), C.byref(out)), "npd_workspace_bytes")
+    return out.value
+
+
+def npd_kd_fwd_bwd(args: npd_kd_args, stream=None) -> None:
+    _check(lib().npd_kd_fwd_bwd(C.byref(args), _stream(stream)), "npd_kd_fwd_bwd")
+
+
+def npd_kd_fwd_bwd_host(host: npd_kd_args, dev: npd_kd_args, stream=None) -> None:
+    _check(lib().npd_kd_fwd_bwd_host(C.byref(host), C.byref(dev), _stream(stream)), "npd_kd_fwd_bwd_host")
+
+
+def npd_last_status(workspace: torch.Tensor, stream=None) -> int:
+    out = C.c_int32(0)
+    _check(lib().npd_last_status(workspace.data_ptr(), _stream(stream), C.byref(out)), "npd_last_status")
+    return out.value
+
+
+def npd_last_launch_count() -> int:
+    return lib().npd_last_launch_count()
+
+
+def npd_segment_stats(cu_seqlens, loss_mask, labels, kl, nll_student, nll_teacher, *,
+                      kl_sum=None, nll_s_sum=None, nll_t_sum=None, count=None, seg_id=None,
+                      status=None, stream=None):
+    """Per-segment sums and counts.  Allocates the outputs that are not given and
+    returns (kl_sum, nll_s_sum, nll_t_sum, count, seg_id)."""
+    S = cu_seqlens.numel() - 1
+    ref = next(t for t in (kl, nll_student, nll_teacher, loss_mask, labels, cu_seqlens) if t is not None)
+    T = ref.numel() if ref is not cu_seqlens else int(cu_seqlens[-1].item())
+    dev = cu_seqlens.device
+    f = lambda src, out: (torch.empty(S, dtype=torch.float32, device=dev) if out is None and src is not None else out)
+    kl_sum, nll_s_sum, nll_t_sum = f(kl, kl_sum), f(nll_student, nll_s_sum), f(nll_teacher, nll_t_sum)
+    if count is None:
+        count = torch.empty(S, dtype=torch.int32, device=dev)
+    if seg_id is None:
+        seg_id = torch.empty(T, dtype=torch.int32, device=dev)
+    _check(lib().npd_segment_stats(T, S, _ptr(cu_seqlens), _ptr(loss_mask), _ptr(labels), _ptr(kl),
+                                   _ptr(nll_student), _ptr(nll_teacher), _ptr(kl_sum), _ptr(nll_s_sum),
+                                   _ptr(nll_t_sum), _ptr(count), _ptr(seg_id), _ptr(status),
+                                   _stream(stream)), "npd_segment_stats")
+    return kl_sum, nll_s_sum, nll_t_sum, count, seg_id
+
+
+def npd_select(cond_seg, uncond_seg, nll_s_sum, nll_t_sum, count, lo: float, hi: float, flags: int = 0,
+               stream=None):
+    """Delta-IFD scores and keep mask.  Returns (ifd_teacher, ifd_student, delta, keep, n_keep)."""
+    N, S, dev = cond_seg.numel(), count.numel(), cond_seg.device
+    ifd_t = torch.empty(N, dtype=torch.float32, device=dev)
+    ifd_s = torch.empty(N, dtype=torch.float32, device=dev)
+    delta = torch.empty(N, dtype=torch.float32, device=dev)
+    keep = torch.empty(N, dtype=torch.uint8, device=dev)
+    n_keep = torch.empty(1, dtype=torch.int32, device=dev)
+    _check(lib().npd_select(N, _ptr(cond_seg), _ptr(uncond_seg), _ptr(nll_s_sum), _ptr(nll_t_sum),
+                            _ptr(count), S, float(lo), float(hi), int(flags), _ptr(ifd_t), _ptr(ifd_s),
+                            _ptr(delta), _ptr(keep), _ptr(n_keep), _stream(stream)), "npd_select")
+    return ifd_t, ifd_s, delta, keep, n_keep
+
+
+def npd_gemm_bf16(A, B, out, *, a_mn_major=False, b_mn_major=False, out_mode=NPD_GEMM_STORE_F32,
+                  k_splits=1, stream=None):
+    """out[M,N] (+)= sum_k A[m,k] B[n,k].  A is [M,K] (K-major) or [K,M] (MN-major); same for B."""
+    M, N = out.shape
+    K = A.shape[0] if a_mn_major else A.shape[1]
+    _check(lib().npd_gemm_bf16(M, N, K, _ptr(A), A.stride(0), int(a_mn_major), _ptr(B), B.stride(0),
+                               int(b_mn_major), _ptr(out), out.stride(0), int(out_mode), int(k_splits),
+                               _stream(stream)), "npd_gemm_bf16")
+    return out
+
+
+class KDStep:
+    """Holds the output and workspace tensors of one problem shape and runs the
+    fused step on them; a convenience over the raw calls."""
+
+    def __init__(self, batch, *, grads=True, dw_dtype=torch.bfloat16, grad_chunk_cols=0, grad_scale=None):
+        dev = batch.hidden.device
+        T, d, V = batch.T, batch.d, batch.V
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.batch = batch
+        self.kl = torch.empty(T, **f32)
+        self.nll_student = torch.empty(T, **f32)
+        self.nll_teacher = torch.empty(T, **f32)
+        self.d_hidden = torch.empty((T, d), dtype=torch.bfloat16, device=dev) if grads else None
+        self.d_weight = torch.empty((V, d), dtype=dw_dtype, device=dev) if grads else None
+        self.grad_scale = (1.0 / max(batch.n_loss, 1)) if grad_scale is None else grad_scale
+        self._kw = dict(cu_seqlens=batch.cu_seqlens, loss_mask=batch.loss_mask, labels=batch.labels,
+                        temperature=batch.tau, grad_scale=self.grad_scale, kl=self.kl,
+                        nll_student=self.nll_student, nll_teacher=self.nll_teacher,
+                        d_hidden=self.d_hidden, d_weight=self.d_weight, grad_chunk_cols=grad_chunk_cols)
+        probe = make_kd_args(batch.hidden, batch.weight, batch.teacher, **self._kw)
+        nbytes = npd_workspace_bytes(probe)
+        self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
+        off = (-self.workspace.data_ptr()) % 1024
+        self._ws_view = self.workspace[off: off + nbytes]
+        self.args = make_kd_args(batch.hidden, batch.weight, batch.teacher, workspace=self._ws_view,
+                                 **self._kw)
+
+    def run(self, stream=None):
+        npd_kd_fwd_bwd(self.args, stream)
+
+    def status(self, stream=None) -> int:
+        return npd_last_status(self._ws_view, stream)

@@ -1,0 +1,379 @@
+// Fused LM-head tile kernel of the distillation step.
+//
+// For a 128-token row block and a run of 256-wide vocabulary tiles it forms the
+// student logits O_S = H W^T (Algorithm 1, "Compute Student Logits") on
+// tcgen05 tensor cores with the accumulator in tensor memory, streams the
+// matching teacher-logit tile O_T through shared memory with TMA, and consumes
+// both on chip.  The T x V logits are never written to global memory.
+//
+//   kForward : online softmax statistics of Softmax(O_T/tau) and Softmax(O_S/tau)
+//              (Algorithm 1, "Compute Probs") and the cross term of Eq. 2, kept
+//              as running (max, sum, sum*(difference)) per token and written as
+//              partial results per vocabulary split.
+//   kGradient: with the per-token log-sum-exps known, the logit gradient
+//              dO_S = coef_t (p_S - p_T), coef_t = grad_scale*m_t/tau (gradient of
+//              Eq. 2), rounded to bf16 and stored to a scratch block that the two
+//              backward contractions read.
+//
+// CTA = 384 threads, one CTA per SM, persistent over work units:
+//   warp 0      TMA producer for the H and W operand stages (3-stage ring)
+//   warp 1      tcgen05.mma issuer; owns the 512 TMEM columns (2 accumulators 128x256)
+//   warp 2      TMA producer for the teacher sub-tiles (two 2-stage rings)
+//   warps 4-11  epilogue; warp w reads TMEM lanes 32*(w%4).., columns 128*((w-4)/4)..
+//               so every thread owns one token row and half of the tile's columns.
+// All exponentials are taken in base 2 on logits pre-scaled by log2(e)/tau.
+#pragma once
+
+#include "ptx_sm100.cuh"
+
+namespace npd {
+
+enum KdTileMode : int { kForward = 0, kGradient = 1 };
+
+// Per-token fields of a forward partial (one partial per vocabulary split and column half).
+enum : int { kPMaxA = 0, kPSumA, kPCross, kPMaxB, kPSumB, kPSumA1, kPSumB1, kPFields };
+
+struct KdTileParams {
+  int T, V;
+  int ksteps;       // d / 64
+  int row_blocks;   // ceil(T / 128)
+  int vt_begin;     // first 256-wide vocabulary tile of this launch
+  int vt_count;     // number of vocabulary tiles of this launch
+  int nsplit;       // the vt_count tiles are cut into nsplit runs; a unit = (row block, run)
+  float scale2;     // log2(e) / tau
+  float tau;
+  // forward
+  float* partials;  // [2*nsplit][kPFields][T]
+  // gradient
+  const float* lse2_a;  // [T] log2-sum-exp2 of the scaled teacher logits
+  const float* lse2_b;  // [T] same for the student
+  const float* coef;    // [T] grad_scale * m_t / tau
+  int g_col0;           // vocabulary column that scratch column 0 holds
+  int* status;
+};
+
+namespace kd_cfg {
+constexpr int BM = 128, BN = 256, BK = 64, UK = 16;
+constexpr int STAGES = 3;
+constexpr int A_BYTES = BM * BK * 2;       // 16 KB
+constexpr int B_BYTES = BN * BK * 2;       // 32 KB
+constexpr int ZSUB_COLS = 64;              // teacher sub-tile: 128 rows x 64 bf16 (128 B rows)
+constexpr int ZSUB_BYTES = BM * ZSUB_COLS * 2;  // 16 KB
+constexpr int ZQ = 2;                      // ring depth per column half
+constexpr int THREADS = 384;
+constexpr int TMEM_COLS = 512;
+constexpr int OFF_A = 0;
+constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
+constexpr int OFF_Z = OFF_B + STAGES * B_BYTES;
+constexpr int OFF_BAR = OFF_Z + 2 * ZQ * ZSUB_BYTES;
+constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * ZQ;
+constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;
+constexpr float kNegClamp = -1.0e30f;      // finite stand-in for -inf teacher logits
+}  // namespace kd_cfg
+
+template <int kMode, bool kTauIsOne>
+__global__ void __launch_bounds__(kd_cfg::THREADS, 1)
+kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
+               const __grid_constant__ CUtensorMap tmap_t, const __grid_constant__ CUtensorMap tmap_g,
+               const KdTileParams p) {
+  using namespace kd_cfg;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~static_cast<uintptr_t>(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t full0 = smem_u32(bars);
+  const uint32_t empty0 = full0 + 8 * STAGES;
+  const uint32_t tfull0 = empty0 + 8 * STAGES;
+  const uint32_t tempty0 = tfull0 + 16;
+  const uint32_t zfull0 = tempty0 + 16;           // [half][ZQ]
+  const uint32_t zempty0 = zfull0 + 8 * 2 * ZQ;   // [half][ZQ]
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(tfull0 + 8 * b, 1);
+      mbar_init(tempty0 + 8 * b, 8);
+    }
+    for (int i = 0; i < 2 * ZQ; ++i) {
+      mbar_init(zfull0 + 8 * i, 1);
+      mbar_init(zempty0 + 8 * i, kMode == kForward ? 4 : 1);
+    }
+    *abort_flag = 0;
+    fence_mbar_init();
+    prefetch_tmap(&tmap_h);
+    prefetch_tmap(&tmap_w);
+    prefetch_tmap(&tmap_t);
+    if (kMode == kGradient) prefetch_tmap(&tmap_g);
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int units = p.row_blocks * p.nsplit;
+  auto run_of = [&](int u, int& r, int& s, int& vt0, int& vt1) {
+    r = u % p.row_blocks;
+    s = u / p.row_blocks;
+    vt0 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * s / p.nsplit);
+    vt1 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * (s + 1) / p.nsplit);
+  };
+
+  if (warp == 0) {
+    // ---------------------- operand producer (H and W stages) ----------------------
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        int r, s, vt0, vt1;
+        run_of(u, r, s, vt0, vt1);
+        for (int vt = vt0; vt < vt1 && ok; ++vt) {
+          for (int ks = 0; ks < p.ksteps; ++ks, ++it) {
+            const uint32_t st = it % STAGES, ph = (it / STAGES) & 1;
+            if (!(ok = mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag))) break;
+            const uint32_t fb = full0 + 8 * st;
+            mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
+            tma_load_2d(smem_u32(smem + OFF_A + st * A_BYTES), &tmap_h, fb, ks * BK, r * BM);
+            tma_load_2d(smem_u32(smem + OFF_B + st * B_BYTES), &tmap_w, fb, ks * BK, vt * BN);
+          }
+        }
+      }
+      const uint32_t last = it < STAGES ? it : STAGES;
+      for (uint32_t j = 0; j < last; ++j) {
+        const uint32_t i2 = it - 1 - j;
+        mbar_wait(full0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1, abort_flag);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------- MMA issuer ----------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, false, false);
+      uint32_t it = 0, tile = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        int r, s, vt0, vt1;
+        run_of(u, r, s, vt0, vt1);
+        for (int vt = vt0; vt < vt1 && ok; ++vt, ++tile) {
+          const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
+          if (!(ok = mbar_wait(tempty0 + 8 * buf, tph ^ 1, abort_flag))) break;
+          tc_fence_after_sync();
+          const uint32_t d_tmem = tmem_base + buf * BN;
+          for (int ks = 0; ks < p.ksteps; ++ks, ++it) {
+            const uint32_t st = it % STAGES, ph = (it / STAGES) & 1;
+            if (!(ok = mbar_wait(full0 + 8 * st, ph, abort_flag))) break;
+            tc_fence_after_sync();
+            const uint32_t sa = smem_u32(smem + OFF_A + st * A_BYTES);
+            const uint32_t sb = smem_u32(smem + OFF_B + st * B_BYTES);
+#pragma unroll
+            for (int k = 0; k < BK / UK; ++k) {
+              umma_bf16(d_tmem, umma_desc_sw128(sa + k * (UK * 2), 16, 1024),
+                        umma_desc_sw128(sb + k * (UK * 2), 16, 1024), idesc, (ks > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(empty0 + 8 * st);
+          }
+          if (ok) umma_commit(tfull0 + 8 * buf);
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ---------------------- teacher producer ----------------------
+    if (lane == 0) {
+      uint32_t zit = 0;  // sub-tile pairs issued; both halves advance together
+      bool ok = true;
+      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+        int r, s, vt0, vt1;
+        run_of(u, r, s, vt0, vt1);
+        for (int vt = vt0; vt < vt1 && ok; ++vt) {
+          for (int j = 0; j < BN / 2 / ZSUB_COLS && ok; ++j, ++zit) {
+            const uint32_t q = zit % ZQ, ph = (zit / ZQ) & 1;
+            for (int half = 0; half < 2; ++half) {
+              const int col = vt * BN + half * (BN / 2) + j * ZSUB_COLS;
+              const uint32_t bi = 8 * (half * ZQ + q);
+              if (!(ok = mbar_wait(zempty0 + bi, ph ^ 1, abort_flag))) break;
+              mbar_arrive_expect_tx(zfull0 + bi, ZSUB_BYTES);
+              tma_load_2d(smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES), &tmap_t, zfull0 + bi,
+                          col, r * BM);
+            }
+          }
+        }
+      }
+      const uint32_t last = zit < ZQ ? zit : ZQ;
+      for (uint32_t j = 0; j < last; ++j) {
+        const uint32_t i2 = zit - 1 - j;
+        for (int half = 0; half < 2; ++half)
+          mbar_wait(zfull0 + 8 * (half * ZQ + (i2 % ZQ)), (i2 / ZQ) & 1, abort_flag);
+      }
+    }
+  } else if (warp >= 4) {
+    // ---------------------- epilogue ----------------------
+    const int e = warp - 4;
+    const int lg = e & 3;      // == warp % 4: the TMEM lane group this warp may read
+    const int half = e >> 2;   // which 128 columns of the 256-wide tile
+    const int row_local = lg * 32 + lane;
+    const uint32_t swz = static_cast<uint32_t>(row_local & 7);
+    uint32_t tile = 0, zit = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      int r, s, vt0, vt1;
+      run_of(u, r, s, vt0, vt1);
+      const int row = r * BM + row_local;
+      // forward state (base-2 domain): running max / sum of the scaled teacher (a) and student (b)
+      float m_a = -INFINITY, s_a = 0.f, cross = 0.f, m_b = -INFINITY, s_b = 0.f, s_a1 = 0.f, s_b1 = 0.f;
+      float g_lse_a = 0.f, g_lse_b = 0.f, g_coef = 0.f;
+      if (kMode == kGradient && row < p.T) {
+        g_lse_a = p.lse2_a[row];
+        g_lse_b = p.lse2_b[row];
+        g_coef = p.coef[row];
+      }
+      for (int vt = vt0; vt < vt1 && ok; ++vt, ++tile) {
+        const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * buf, tph, abort_flag));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t taddr =
+            tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN + half * (BN / 2);
+        for (int j = 0; j < BN / 2 / ZSUB_COLS && ok; ++j, ++zit) {
+          const uint32_t q = zit % ZQ, zph = (zit / ZQ) & 1;
+          const uint32_t bi = 8 * (half * ZQ + q);
+          ok = __all_sync(0xffffffffu, mbar_wait(zfull0 + bi, zph, abort_flag));
+          if (!ok) break;
+          uint8_t* zrow = smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES + row_local * 128;
+          const int sub_col0 = vt * BN + half * (BN / 2) + j * ZSUB_COLS;
+#pragma unroll 1
+          for (int c = 0; c < ZSUB_COLS / 32; ++c) {
+            const int col0 = sub_col0 + c * 32;
+            uint32_t acc[32];
+            tmem_ld32(taddr + j * ZSUB_COLS + c * 32, acc);
+            uint4 zq[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              zq[i] = *reinterpret_cast<const uint4*>(zrow + ((static_cast<uint32_t>(c * 4 + i) ^ swz) << 4));
+            tmem_ld_wait();
+            const int nvalid = p.V - col0;  // columns of this chunk inside the vocabulary
+            float zt[32];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t w[4] = {zq[i].x, zq[i].y, zq[i].z, zq[i].w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                zt[8 * i + 2 * k] = fmaxf(bf16_lo(w[k]), kNegClamp);
+                zt[8 * i + 2 * k + 1] = fmaxf(bf16_hi(w[k]), kNegClamp);
+              }
+            }
+            if (kMode == kForward) {
+              if (nvalid > 0) {
+                float zs[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) zs[i] = __uint_as_float(acc[i]);
+                if (nvalid < 32) {
+#pragma unroll
+                  for (int i = 0; i < 32; ++i)
+                    if (i >= nvalid) { zs[i] = kNegClamp; zt[i] = kNegClamp; }
+                }
+                float ca = zt[0], cb = zs[0];
+#pragma unroll
+                for (int i = 1; i < 32; ++i) { ca = fmaxf(ca, zt[i]); cb = fmaxf(cb, zs[i]); }
+                ca *= p.scale2;
+                cb *= p.scale2;
+                if (ca > m_a) {
+                  const float f = ex2f(m_a - ca);
+                  s_a *= f;
+                  cross *= f;
+                  if (!kTauIsOne) s_a1 *= ex2f((m_a - ca) * p.tau);
+                  m_a = ca;
+                }
+                if (cb > m_b) {
+                  s_b *= ex2f(m_b - cb);
+                  if (!kTauIsOne) s_b1 *= ex2f((m_b - cb) * p.tau);
+                  m_b = cb;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                  const float ta = fmaf(zt[i], p.scale2, -m_a);
+                  const float tb = fmaf(zs[i], p.scale2, -m_b);
+                  const float ea = ex2f(ta);
+                  s_a += ea;
+                  cross = fmaf(ea, zt[i] - zs[i], cross);
+                  s_b += ex2f(tb);
+                  if (!kTauIsOne) {
+                    s_a1 += ex2f(ta * p.tau);
+                    s_b1 += ex2f(tb * p.tau);
+                  }
+                }
+              }
+            } else {
+              // gradient tile: dO_S = coef * (p_S - p_T), written back in place over the teacher
+              uint32_t packed[16];
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                float g0 = g_coef * (ex2f(fmaf(__uint_as_float(acc[i]), p.scale2, -g_lse_b)) -
+                                     ex2f(fmaf(zt[i], p.scale2, -g_lse_a)));
+                float g1 = g_coef * (ex2f(fmaf(__uint_as_float(acc[i + 1]), p.scale2, -g_lse_b)) -
+                                     ex2f(fmaf(zt[i + 1], p.scale2, -g_lse_a)));
+                if (i >= nvalid) g0 = 0.f;
+                if (i + 1 >= nvalid) g1 = 0.f;
+                packed[i >> 1] = pack_bf16x2(g0, g1);
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                *reinterpret_cast<uint4*>(zrow + ((static_cast<uint32_t>(c * 4 + i) ^ swz) << 4)) =
+                    make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+            }
+          }
+          if (kMode == kForward) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(zempty0 + bi);
+          } else {
+            // hand the finished 128 x 64 gradient sub-tile to TMA, then recycle the stage
+            fence_proxy_async_smem();
+            named_barrier_sync(1 + half, 128);
+            if (lg == 0 && lane == 0) {
+              tma_store_2d(&tmap_g, smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES),
+                           sub_col0 - p.g_col0, r * BM);
+              tma_store_commit();
+              tma_store_wait_read<0>();
+              mbar_arrive(zempty0 + bi);
+            }
+          }
+        }
+        if (!ok) break;
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty0 + 8 * buf);
+      }
+      if (kMode == kForward && ok && row < p.T) {
+        float* dst = p.partials + (static_cast<size_t>(2 * s + half) * kPFields) * p.T + row;
+        dst[static_cast<size_t>(kPMaxA) * p.T] = m_a;
+        dst[static_cast<size_t>(kPSumA) * p.T] = s_a;
+        dst[static_cast<size_t>(kPCross) * p.T] = cross;
+        dst[static_cast<size_t>(kPMaxB) * p.T] = m_b;
+        dst[static_cast<size_t>(kPSumB) * p.T] = s_b;
+        if (!kTauIsOne) {
+          dst[static_cast<size_t>(kPSumA1) * p.T] = s_a1;
+          dst[static_cast<size_t>(kPSumB1) * p.T] = s_b1;
+        }
+      }
+    }
+    if (kMode == kGradient && lg == 0 && lane == 0) tma_store_wait_all<0>();
+  }
+
+  // ---------------------- teardown ----------------------
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && *abort_flag != 0 && p.status != nullptr) atomicCAS(p.status, 0, kStatusTimeout);
+}
+
+}  // namespace npd

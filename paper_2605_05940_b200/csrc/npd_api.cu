@@ -1,0 +1,476 @@
+// Host side of the C ABI declared in include/npd.h: argument checks, workspace
+// layout, TMA descriptors and kernel launches.  Nothing here allocates device
+// memory or keeps state between calls.
+#include "../../include/npd.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+#include "gemm_sm100.cuh"
+#include "kd_tile_sm100.cuh"
+#include "small_kernels.cuh"
+
+namespace {
+
+using namespace npd;
+
+thread_local int g_launches = 0;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+PFN_cuTensorMapEncodeTiled_v12000 tensor_map_encoder() {
+  static PFN_cuTensorMapEncodeTiled_v12000 fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(f);
+  }();
+  return fn;
+}
+
+// 2-D bf16 tensor map with 128-byte swizzle.  inner = contiguous extent (elements),
+// outer = rows, ld = row stride (elements), box = {box_inner (64), box_outer}.
+bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t ld,
+              uint32_t box_inner, uint32_t box_outer) {
+  auto enc = tensor_map_encoder();
+  if (enc == nullptr) return false;
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct DeviceInfo {
+  int sms = 0;
+  int cc_major = 0;
+};
+int device_info(DeviceInfo* out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return NPD_ECUDA;
+  if (cudaDeviceGetAttribute(&out->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&out->cc_major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+    return NPD_ECUDA;
+  return NPD_OK;
+}
+
+// How many runs to cut the vocabulary tiles into so that row_blocks * nsplit work
+// units spread evenly over the SMs.  Cost = rounds of units x tiles per unit.
+int choose_nsplit(int row_blocks, int vtiles, int sms) {
+  int best = 1;
+  long long best_cost = -1;
+  const int max_split = std::min(vtiles, 128);
+  for (int ns = 1; ns <= max_split; ++ns) {
+    const long long rounds = (static_cast<long long>(row_blocks) * ns + sms - 1) / sms;
+    const long long per = (vtiles + ns - 1) / ns;
+    const long long cost = rounds * per * 64 + ns;  // small bias towards fewer splits
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best = ns;
+    }
+  }
+  return best;
+}
+
+struct Plan {
+  int row_blocks, vtiles, nsplit, nslots;
+  int chunk_cols;     // vocabulary columns per gradient chunk (multiple of 256)
+  int nchunks;
+  bool grads;
+  size_t off_status, off_partials, off_lse_a, off_lse_b, off_coef, off_g, off_dh, total;
+};
+
+int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
+  pl->row_blocks = (a->T + 127) / 128;
+  pl->vtiles = (a->V + 255) / 256;
+  pl->nsplit = choose_nsplit(pl->row_blocks, pl->vtiles, sms);
+  pl->nslots = 2 * pl->nsplit;
+  pl->grads = a->d_hidden != nullptr || a->d_weight != nullptr;
+  const int vpad = pl->vtiles * 256;
+  int cc = a->grad_chunk_cols > 0 ? a->grad_chunk_cols : 4096;
+  cc = std::min((cc + 255) / 256 * 256, vpad);
+  pl->chunk_cols = cc;
+  pl->nchunks = (vpad + cc - 1) / cc;
+  size_t off = 0;
+  pl->off_status = off;
+  off += 1024;
+  pl->off_partials = off;
+  off = align_up(off + sizeof(float) * pl->nslots * kPFields * static_cast<size_t>(a->T), 1024);
+  pl->off_lse_a = off;
+  off = align_up(off + sizeof(float) * a->T, 1024);
+  pl->off_lse_b = off;
+  off = align_up(off + sizeof(float) * a->T, 1024);
+  pl->off_coef = off;
+  off = align_up(off + sizeof(float) * a->T, 1024);
+  pl->off_g = off;
+  pl->off_dh = off;
+  if (pl->grads) {
+    off = align_up(off + 2 * static_cast<size_t>(a->T) * cc, 1024);
+    pl->off_dh = off;
+    if (pl->nchunks > 1) off = align_up(off + sizeof(float) * static_cast<size_t>(a->T) * a->d, 1024);
+  }
+  pl->total = off;
+  return NPD_OK;
+}
+
+int check_args(const npd_kd_args* a, bool need_pointers) {
+  if (a == nullptr || a->size != sizeof(npd_kd_args)) return NPD_EINVAL;
+  if (a->T < 1 || a->d < 1 || a->V < 1) return NPD_EINVAL;
+  if (!(a->temperature > 0.f) || !std::isfinite(a->temperature)) return NPD_EINVAL;
+  if (a->teacher_dtype == NPD_DTYPE_F32) return NPD_EUNSUPPORTED;
+  if (a->teacher_dtype != NPD_DTYPE_BF16) return NPD_EINVAL;
+  if (a->d_weight_dtype != NPD_DTYPE_BF16 && a->d_weight_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
+  if (a->grad_chunk_cols < 0) return NPD_EINVAL;
+  if (a->d % 64 != 0) return NPD_ESHAPE;
+  if (a->ldh < a->d || a->ldw < a->d || a->ldt < a->V) return NPD_ESHAPE;
+  if (a->cu_seqlens != nullptr && (a->S < 1 || a->S > a->T)) return NPD_ESHAPE;
+  if ((a->ldh % 8) || (a->ldw % 8) || (a->ldt % 8)) return NPD_EALIGN;
+  if ((a->d_hidden == nullptr) != (a->d_weight == nullptr)) return NPD_EINVAL;
+  if ((a->flags & NPD_KD_ACCUMULATE_DW) && a->d_weight_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
+  if (!need_pointers) return NPD_OK;
+  if (a->hidden == nullptr || a->weight == nullptr || a->teacher == nullptr || a->kl == nullptr)
+    return NPD_EINVAL;
+  if (!aligned16(a->hidden) || !aligned16(a->weight) || !aligned16(a->teacher) ||
+      !aligned16(a->d_hidden) || !aligned16(a->d_weight))
+    return NPD_EALIGN;
+  if (a->d_weight != nullptr && a->d_weight_dtype == NPD_DTYPE_F32 && (a->ldw % 4)) return NPD_EALIGN;
+  return NPD_OK;
+}
+
+template <typename K>
+int set_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess
+             ? NPD_OK
+             : NPD_ECUDA;
+}
+
+int launch_gemm(bool a_mn, bool b_mn, const void* A, long long lda, const void* B, long long ldb,
+                const GemmParams& gp, int sms, cudaStream_t st) {
+  using namespace gemm_cfg;
+  CUtensorMap ma, mb;
+  const bool oka = a_mn ? make_map(&ma, A, gp.M, gp.K, lda, 64, 64) : make_map(&ma, A, gp.K, gp.M, lda, 64, BM);
+  const bool okb = b_mn ? make_map(&mb, B, gp.N, gp.K, ldb, 64, 64) : make_map(&mb, B, gp.K, gp.N, ldb, 64, BN);
+  if (!oka || !okb) return NPD_ECUDA;
+  const int units = ((gp.M + BM - 1) / BM) * ((gp.N + BN - 1) / BN) * gp.k_splits;
+  const int grid = std::min(units, sms);
+  void (*k)(const CUtensorMap, const CUtensorMap, const GemmParams) = nullptr;
+  if (!a_mn && !b_mn) k = gemm_bf16_kernel<false, false>;
+  if (!a_mn && b_mn) k = gemm_bf16_kernel<false, true>;
+  if (a_mn && !b_mn) k = gemm_bf16_kernel<true, false>;
+  if (a_mn && b_mn) k = gemm_bf16_kernel<true, true>;
+  if (set_smem(k, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
+  k<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, gp);
+  ++g_launches;
+  return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
+}
+
+template <int kMode>
+int launch_kd_tile(bool tau_one, const CUtensorMap& mh, const CUtensorMap& mw, const CUtensorMap& mt,
+                   const CUtensorMap& mg, const KdTileParams& kp, int sms, cudaStream_t st) {
+  using namespace kd_cfg;
+  auto k = tau_one ? kd_tile_kernel<kMode, true> : kd_tile_kernel<kMode, false>;
+  if (set_smem(k, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
+  const int units = kp.row_blocks * kp.nsplit;
+  k<<<std::min(units, sms), THREADS, SMEM_BYTES, st>>>(mh, mw, mt, mg, kp);
+  ++g_launches;
+  return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* npd_strerror(int status) {
+  switch (status) {
+    case NPD_OK: return "ok";
+    case NPD_EINVAL: return "invalid argument";
+    case NPD_ESHAPE: return "unsupported shape or stride";
+    case NPD_EALIGN: return "pointer or stride not 16-byte aligned";
+    case NPD_ESEQ: return "malformed cu_seqlens";
+    case NPD_EARCH: return "device is not compute capability 10.x";
+    case NPD_EWORKSPACE: return "workspace missing, misaligned or too small";
+    case NPD_ECUDA: return "CUDA call failed";
+    case NPD_ETIMEOUT: return "bounded device-side wait expired";
+    case NPD_EUNSUPPORTED: return "option not implemented";
+    default: return "unknown status";
+  }
+}
+
+int npd_last_launch_count(void) { return g_launches; }
+
+int npd_workspace_bytes(const npd_kd_args* args, size_t* out_bytes) {
+  if (out_bytes == nullptr) return NPD_EINVAL;
+  int rc = check_args(args, false);
+  if (rc != NPD_OK) return rc;
+  DeviceInfo di;
+  if ((rc = device_info(&di)) != NPD_OK) return rc;
+  Plan pl;
+  make_plan(args, di.sms, &pl);
+  *out_bytes = pl.total;
+  return NPD_OK;
+}
+
+int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
+  g_launches = 0;
+  int rc = check_args(a, true);
+  if (rc != NPD_OK) return rc;
+  DeviceInfo di;
+  if ((rc = device_info(&di)) != NPD_OK) return rc;
+  if (di.cc_major != 10) return NPD_EARCH;
+  Plan pl;
+  make_plan(a, di.sms, &pl);
+  if (a->workspace == nullptr || (reinterpret_cast<uintptr_t>(a->workspace) & 1023u) ||
+      a->workspace_bytes < pl.total)
+    return NPD_EWORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  uint8_t* ws = static_cast<uint8_t*>(a->workspace);
+  int* status = reinterpret_cast<int*>(ws + pl.off_status);
+  float* partials = reinterpret_cast<float*>(ws + pl.off_partials);
+  float* lse_a = reinterpret_cast<float*>(ws + pl.off_lse_a);
+  float* lse_b = reinterpret_cast<float*>(ws + pl.off_lse_b);
+  float* coef = reinterpret_cast<float*>(ws + pl.off_coef);
+  if (cudaMemsetAsync(status, 0, 64, st) != cudaSuccess) return NPD_ECUDA;
+
+  const bool tau_one = a->temperature == 1.0f;
+  const float scale2 = 1.4426950408889634f / a->temperature;
+
+  CUtensorMap mh, mw, mt;
+  if (!make_map(&mh, a->hidden, a->d, a->T, a->ldh, 64, 128) ||
+      !make_map(&mw, a->weight, a->d, a->V, a->ldw, 64, 256) ||
+      !make_map(&mt, a->teacher, a->V, a->T, a->ldt, 64, 128))
+    return NPD_ECUDA;
+
+  // cu_seqlens is validated on the device; the result lands in the status word.
+  if (a->cu_seqlens != nullptr) {
+    segment_stats_kernel<<<(a->S + 3) / 4, 128, 0, st>>>(a->T, a->S, a->cu_seqlens, nullptr, nullptr,
+                                                        nullptr, nullptr, nullptr, nullptr, nullptr,
+                                                        nullptr, nullptr, nullptr, status);
+    ++g_launches;
+  }
+
+  // ---- forward: statistics per (row block, vocabulary run), then the per-token merge ----
+  KdTileParams kp{};
+  kp.T = a->T;
+  kp.V = a->V;
+  kp.ksteps = a->d / 64;
+  kp.row_blocks = pl.row_blocks;
+  kp.vt_begin = 0;
+  kp.vt_count = pl.vtiles;
+  kp.nsplit = pl.nsplit;
+  kp.scale2 = scale2;
+  kp.tau = a->temperature;
+  kp.partials = partials;
+  kp.status = status;
+  if ((rc = launch_kd_tile<kForward>(tau_one, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
+
+  CombineParams cp{};
+  cp.T = a->T;
+  cp.d = a->d;
+  cp.V = a->V;
+  cp.nslots = pl.nslots;
+  cp.partials = partials;
+  cp.hidden = static_cast<const __nv_bfloat16*>(a->hidden);
+  cp.weight = static_cast<const __nv_bfloat16*>(a->weight);
+  cp.teacher = static_cast<const __nv_bfloat16*>(a->teacher);
+  cp.ldh = a->ldh;
+  cp.ldw = a->ldw;
+  cp.ldt = a->ldt;
+  cp.loss_mask = a->loss_mask;
+  cp.labels = a->labels;
+  cp.scale2 = scale2;
+  cp.tau = a->temperature;
+  cp.grad_scale = a->grad_scale;
+  cp.kl = a->kl;
+  cp.nll_s = a->nll_student;
+  cp.nll_t = a->nll_teacher;
+  cp.lse2_a = lse_a;
+  cp.lse2_b = lse_b;
+  cp.coef = coef;
+  if (tau_one)
+    kd_combine_kernel<true><<<(a->T + 7) / 8, 256, 0, st>>>(cp);
+  else
+    kd_combine_kernel<false><<<(a->T + 7) / 8, 256, 0, st>>>(cp);
+  ++g_launches;
+  if (cudaGetLastError() != cudaSuccess) return NPD_ECUDA;
+  if (!pl.grads) return NPD_OK;
+
+  // ---- backward: per vocabulary chunk, gradient tiles -> scratch -> dW rows and dH partial ----
+  __nv_bfloat16* gbuf = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_g);
+  float* dh_acc = reinterpret_cast<float*>(ws + pl.off_dh);
+  const long long ldg = pl.chunk_cols;
+  for (int c = 0; c < pl.nchunks; ++c) {
+    const int col0 = c * pl.chunk_cols;
+    const int cols = std::min(pl.chunk_cols, a->V - col0);  // columns of this chunk inside V
+    if (cols <= 0) break;
+    const int cols_pad = std::min(pl.chunk_cols, pl.vtiles * 256 - col0);
+    CUtensorMap mg;
+    if (!make_map(&mg, gbuf, cols_pad, a->T, ldg, 64, 128)) return NPD_ECUDA;
+    KdTileParams gp = kp;
+    gp.vt_begin = col0 / 256;
+    gp.vt_count = cols_pad / 256;
+    gp.nsplit = gp.vt_count;
+    gp.partials = nullptr;
+    gp.lse2_a = lse_a;
+    gp.lse2_b = lse_b;
+    gp.coef = coef;
+    gp.g_col0 = col0;
+    if ((rc = launch_kd_tile<kGradient>(tau_one, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
+
+    // dW[col0 .. col0+cols) = G_chunk^T H       (M = vocabulary rows, N = d, K = T)
+    GemmParams gw{};
+    gw.M = cols;
+    gw.N = a->d;
+    gw.K = a->T;
+    gw.k_splits = 1;
+    gw.ldo = a->ldw;
+    gw.status = status;
+    if (a->d_weight_dtype == NPD_DTYPE_F32) {
+      gw.out = static_cast<float*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw;
+      gw.out_mode = (a->flags & NPD_KD_ACCUMULATE_DW) ? kOutAddF32 : kOutStoreF32;
+    } else {
+      gw.out = static_cast<__nv_bfloat16*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw;
+      gw.out_mode = kOutStoreBF16;
+    }
+    if ((rc = launch_gemm(true, true, gbuf, ldg, a->hidden, a->ldh, gw, di.sms, st)) != NPD_OK) return rc;
+
+    // dH (+)= G_chunk W[col0 .. col0+cols)      (M = T, N = d, K = vocabulary rows of the chunk)
+    GemmParams gh{};
+    gh.M = a->T;
+    gh.N = a->d;
+    gh.K = cols;
+    gh.k_splits = 1;
+    gh.status = status;
+    if (pl.nchunks == 1) {
+      gh.out = a->d_hidden;
+      gh.ldo = a->ldh;
+      gh.out_mode = kOutStoreBF16;
+    } else {
+      gh.out = dh_acc;
+      gh.ldo = a->d;
+      gh.out_mode = c == 0 ? kOutStoreF32 : kOutAddF32;
+    }
+    const __nv_bfloat16* wc = static_cast<const __nv_bfloat16*>(a->weight) + static_cast<size_t>(col0) * a->ldw;
+    if ((rc = launch_gemm(false, true, gbuf, ldg, wc, a->ldw, gh, di.sms, st)) != NPD_OK) return rc;
+  }
+  if (pl.nchunks > 1) {
+    const long long n = static_cast<long long>(a->T) * (a->d / 8);
+    f32_to_bf16_rows_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(
+        dh_acc, a->T, a->d, static_cast<__nv_bfloat16*>(a->d_hidden), a->ldh);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return NPD_ECUDA;
+  }
+  return NPD_OK;
+}
+
+int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* cuda_stream) {
+  if (host == nullptr || dev == nullptr || host->size != sizeof(npd_kd_args)) return NPD_EINVAL;
+  int rc = check_args(dev, true);
+  if (rc != NPD_OK) return rc;
+  if (host->T != dev->T || host->d != dev->d || host->V != dev->V) return NPD_EINVAL;
+  if (host->hidden == nullptr || host->teacher == nullptr || host->kl == nullptr) return NPD_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t T = dev->T;
+  bool ok = true;
+  ok &= cudaMemcpy2DAsync(const_cast<void*>(dev->hidden), dev->ldh * 2, host->hidden, host->ldh * 2,
+                          static_cast<size_t>(dev->d) * 2, T, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpy2DAsync(const_cast<void*>(dev->teacher), dev->ldt * 2, host->teacher, host->ldt * 2,
+                          static_cast<size_t>(dev->V) * 2, T, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (dev->cu_seqlens != nullptr && host->cu_seqlens != nullptr)
+    ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->cu_seqlens), host->cu_seqlens,
+                          sizeof(int32_t) * (dev->S + 1), cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (dev->loss_mask != nullptr && host->loss_mask != nullptr)
+    ok &= cudaMemcpyAsync(const_cast<uint8_t*>(dev->loss_mask), host->loss_mask, T,
+                          cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (dev->labels != nullptr && host->labels != nullptr)
+    ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->labels), host->labels, sizeof(int32_t) * T,
+                          cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) return NPD_ECUDA;
+  if ((rc = npd_kd_fwd_bwd(dev, cuda_stream)) != NPD_OK) return rc;
+  ok &= cudaMemcpyAsync(host->kl, dev->kl, sizeof(float) * T, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (host->nll_student != nullptr && dev->nll_student != nullptr)
+    ok &= cudaMemcpyAsync(host->nll_student, dev->nll_student, sizeof(float) * T,
+                          cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  if (host->nll_teacher != nullptr && dev->nll_teacher != nullptr)
+    ok &= cudaMemcpyAsync(host->nll_teacher, dev->nll_teacher, sizeof(float) * T,
+                          cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  return ok ? NPD_OK : NPD_ECUDA;
+}
+
+int npd_segment_stats(int32_t T, int32_t S, const int32_t* cu_seqlens, const uint8_t* loss_mask,
+                      const int32_t* labels, const float* kl, const float* nll_student,
+                      const float* nll_teacher, float* kl_sum, float* nll_s_sum, float* nll_t_sum,
+                      int32_t* count, int32_t* seg_id, int32_t* status, void* cuda_stream) {
+  if (T < 1 || S < 1 || cu_seqlens == nullptr) return NPD_EINVAL;
+  if (S > T) return NPD_ESHAPE;
+  if ((kl == nullptr) != (kl_sum == nullptr) || (nll_student == nullptr) != (nll_s_sum == nullptr) ||
+      (nll_teacher == nullptr) != (nll_t_sum == nullptr))
+    return NPD_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  segment_stats_kernel<<<(S + 3) / 4, 128, 0, st>>>(T, S, cu_seqlens, loss_mask, labels, kl,
+                                                    nll_student, nll_teacher, kl_sum, nll_s_sum,
+                                                    nll_t_sum, count, seg_id, status);
+  return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
+}
+
+int npd_select(int32_t N, const int32_t* cond_seg, const int32_t* uncond_seg, const float* nll_s_sum,
+               const float* nll_t_sum, const int32_t* count, int32_t S, float lo, float hi,
+               int32_t flags, float* ifd_teacher, float* ifd_student, float* delta, uint8_t* keep,
+               int32_t* n_keep, void* cuda_stream) {
+  if (N < 1 || S < 1 || cond_seg == nullptr || uncond_seg == nullptr || nll_s_sum == nullptr ||
+      nll_t_sum == nullptr || count == nullptr || keep == nullptr || n_keep == nullptr)
+    return NPD_EINVAL;
+  if (std::isnan(lo) || std::isnan(hi)) return NPD_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(n_keep, 0, sizeof(int32_t), st) != cudaSuccess) return NPD_ECUDA;
+  select_kernel<<<(N + 255) / 256, 256, 0, st>>>(N, S, cond_seg, uncond_seg, nll_s_sum, nll_t_sum, count,
+                                                 lo, hi, flags, ifd_teacher, ifd_student, delta, keep,
+                                                 n_keep);
+  return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
+}
+
+int npd_last_status(const void* workspace, void* cuda_stream, int32_t* host_status) {
+  if (workspace == nullptr || host_status == nullptr) return NPD_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(host_status, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return NPD_ECUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? NPD_OK : NPD_ECUDA;
+}
+
+int npd_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32_t a_mn_major,
+                  const void* B, int64_t ldb, int32_t b_mn_major, void* out, int64_t ldo,
+                  int32_t out_mode, int32_t k_splits, void* cuda_stream) {
+  if (M < 1 || N < 1 || K < 1 || A == nullptr || B == nullptr || out == nullptr) return NPD_EINVAL;
+  if (out_mode < kOutStoreF32 || out_mode > kOutAddBF16 || k_splits < 1) return NPD_EINVAL;
+  if (k_splits > 1 && out_mode != kOutAtomicF32) return NPD_EINVAL;
+  if (!aligned16(A) || !aligned16(B) || !aligned16(out) || (lda % 8) || (ldb % 8) || (ldo % 8))
+    return NPD_EALIGN;
+  if (lda < (a_mn_major ? M : K) || ldb < (b_mn_major ? N : K) || ldo < N) return NPD_ESHAPE;
+  DeviceInfo di;
+  int rc = device_info(&di);
+  if (rc != NPD_OK) return rc;
+  if (di.cc_major != 10) return NPD_EARCH;
+  GemmParams gp{};
+  gp.M = M;
+  gp.N = N;
+  gp.K = K;
+  gp.k_splits = k_splits;
+  gp.out = out;
+  gp.ldo = ldo;
+  gp.out_mode = out_mode;
+  gp.status = nullptr;
+  return launch_gemm(a_mn_major != 0, b_mn_major != 0, A, lda, B, ldb, gp, di.sms,
+                     static_cast<cudaStream_t>(cuda_stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,228 @@
+// The per-token and per-sample kernels around the tensor-core tiles: merging the
+// forward partials into losses, segment reductions over cu_seqlens, the Delta-IFD
+// score and selection, and a few layout helpers.  All fp32, deterministic.
+#pragma once
+
+#include "kd_tile_sm100.cuh"
+
+namespace npd {
+
+constexpr float kLn2 = 0.693147180559945309417f;
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ int warp_sum_int(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+struct CombineParams {
+  int T, d, V, nslots;
+  const float* partials;  // [nslots][kPFields][T]
+  const __nv_bfloat16* hidden;
+  const __nv_bfloat16* weight;
+  const __nv_bfloat16* teacher;
+  long long ldh, ldw, ldt;
+  const uint8_t* loss_mask;
+  const int32_t* labels;
+  float scale2, tau, grad_scale;
+  float* kl;
+  float* nll_s;
+  float* nll_t;
+  float* lse2_a;
+  float* lse2_b;
+  float* coef;
+};
+
+// One warp per token.  Merges the per-split online-softmax partials into the token's
+// log-sum-exps, evaluates Eq. 2 as  KL = sum_c p_T(c)(a_c - b_c) - lse(a) + lse(b)
+// (a, b the temperature-scaled teacher / student logits) and the two label
+// cross-entropies behind Eq. 3, and saves what the gradient tiles need.
+template <bool kTauIsOne>
+__global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) {
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= p.T) return;
+  const size_t fs = static_cast<size_t>(p.T);            // field stride
+  const size_t ss = static_cast<size_t>(kPFields) * fs;  // slot stride
+  float ma = -INFINITY, mb = -INFINITY;
+  for (int s = lane; s < p.nslots; s += 32) {
+    const float* q = p.partials + s * ss + t;
+    ma = fmaxf(ma, q[kPMaxA * fs]);
+    mb = fmaxf(mb, q[kPMaxB * fs]);
+  }
+  ma = warp_max(ma);
+  mb = warp_max(mb);
+  float sa = 0.f, cr = 0.f, sb = 0.f, sa1 = 0.f, sb1 = 0.f;
+  for (int s = lane; s < p.nslots; s += 32) {
+    const float* q = p.partials + s * ss + t;
+    const float da = q[kPMaxA * fs] - ma, db = q[kPMaxB * fs] - mb;
+    const float fa = exp2f(da), fb = exp2f(db);
+    sa = fmaf(q[kPSumA * fs], fa, sa);
+    cr = fmaf(q[kPCross * fs], fa, cr);
+    sb = fmaf(q[kPSumB * fs], fb, sb);
+    if (!kTauIsOne) {
+      sa1 = fmaf(q[kPSumA1 * fs], exp2f(da * p.tau), sa1);
+      sb1 = fmaf(q[kPSumB1 * fs], exp2f(db * p.tau), sb1);
+    }
+  }
+  sa = warp_sum(sa);
+  cr = warp_sum(cr);
+  sb = warp_sum(sb);
+  if (!kTauIsOne) {
+    sa1 = warp_sum(sa1);
+    sb1 = warp_sum(sb1);
+  }
+  const float lse_a = ma + log2f(sa), lse_b = mb + log2f(sb);
+  const bool on = p.loss_mask == nullptr || p.loss_mask[t] != 0;
+
+  // label logits: O_S[t, y] = <H[t], W[y]> in fp32, O_T[t, y] read directly
+  float nll_s = 0.f, nll_t = 0.f;
+  if (p.labels != nullptr) {
+    const int y = p.labels[t];
+    if (on && y >= 0 && y < p.V) {
+      const uint4* h4 = reinterpret_cast<const uint4*>(p.hidden + static_cast<size_t>(t) * p.ldh);
+      const uint4* w4 = reinterpret_cast<const uint4*>(p.weight + static_cast<size_t>(y) * p.ldw);
+      float dot = 0.f;
+      for (int i = lane; i < p.d / 8; i += 32) {
+        const uint4 h = h4[i], w = w4[i];
+        dot = fmaf(bf16_lo(h.x), bf16_lo(w.x), dot);
+        dot = fmaf(bf16_hi(h.x), bf16_hi(w.x), dot);
+        dot = fmaf(bf16_lo(h.y), bf16_lo(w.y), dot);
+        dot = fmaf(bf16_hi(h.y), bf16_hi(w.y), dot);
+        dot = fmaf(bf16_lo(h.z), bf16_lo(w.z), dot);
+        dot = fmaf(bf16_hi(h.z), bf16_hi(w.z), dot);
+        dot = fmaf(bf16_lo(h.w), bf16_lo(w.w), dot);
+        dot = fmaf(bf16_hi(h.w), bf16_hi(w.w), dot);
+      }
+      dot = warp_sum(dot);
+      const float zt_y = __bfloat162float(p.teacher[static_cast<size_t>(t) * p.ldt + y]);
+      // natural-log lse of the untempered logits
+      const float nat_b = kTauIsOne ? kLn2 * lse_b : kLn2 * (mb * p.tau + log2f(sb1));
+      const float nat_a = kTauIsOne ? kLn2 * lse_a : kLn2 * (ma * p.tau + log2f(sa1));
+      nll_s = nat_b - dot;
+      nll_t = nat_a - zt_y;
+    }
+  }
+  if (lane == 0) {
+    const float kl = kLn2 * (p.scale2 * (cr / sa) - lse_a + lse_b);
+    p.kl[t] = on ? fmaxf(kl, 0.f) : 0.f;
+    if (p.nll_s != nullptr) p.nll_s[t] = nll_s;
+    if (p.nll_t != nullptr) p.nll_t[t] = nll_t;
+    p.lse2_a[t] = lse_a;
+    p.lse2_b[t] = lse_b;
+    p.coef[t] = on ? p.grad_scale / p.tau : 0.f;
+  }
+}
+
+// One warp per packed segment: masked sums of the per-token values and the count of
+// tokens that carry a label, reduced with warp shuffles in a fixed order; also the
+// token -> segment map and the validation of cu_seqlens.
+__global__ void __launch_bounds__(128) segment_stats_kernel(
+    int T, int S, const int32_t* __restrict__ cu, const uint8_t* __restrict__ mask,
+    const int32_t* __restrict__ labels, const float* __restrict__ kl,
+    const float* __restrict__ nll_s, const float* __restrict__ nll_t, float* kl_sum, float* s_sum,
+    float* t_sum, int32_t* count, int32_t* seg_id, int32_t* status) {
+  const int lane = threadIdx.x & 31;
+  const int s = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (s >= S) return;
+  const int lo = cu[s], hi = cu[s + 1];
+  const bool bad = lo < 0 || hi > T || lo >= hi || (s == 0 && lo != 0) || (s == S - 1 && hi != T);
+  if (bad) {
+    if (lane == 0) {
+      if (status != nullptr) atomicCAS(status, 0, kStatusSeq);
+      if (kl_sum != nullptr) kl_sum[s] = 0.f;
+      if (s_sum != nullptr) s_sum[s] = 0.f;
+      if (t_sum != nullptr) t_sum[s] = 0.f;
+      if (count != nullptr) count[s] = 0;
+    }
+    return;
+  }
+  float a = 0.f, b = 0.f, c = 0.f;
+  int n = 0;
+  for (int t = lo + lane; t < hi; t += 32) {
+    const bool on = mask == nullptr || mask[t] != 0;
+    const bool has = on && (labels == nullptr || labels[t] >= 0);
+    if (on && kl != nullptr) a += kl[t];
+    if (has) {
+      if (nll_s != nullptr) b += nll_s[t];
+      if (nll_t != nullptr) c += nll_t[t];
+      ++n;
+    }
+    if (seg_id != nullptr) seg_id[t] = s;
+  }
+  a = warp_sum(a);
+  b = warp_sum(b);
+  c = warp_sum(c);
+  n = warp_sum_int(n);
+  if (lane == 0) {
+    if (kl_sum != nullptr) kl_sum[s] = a;
+    if (s_sum != nullptr) s_sum[s] = b;
+    if (t_sum != nullptr) t_sum[s] = c;
+    if (count != nullptr) count[s] = n;
+  }
+}
+
+// One thread per sample: IFD (Eq. 3) for teacher and student from token-mean
+// cross-entropies, Delta-IFD (Eq. 4), and the inclusive keep interval.
+__global__ void __launch_bounds__(256) select_kernel(
+    int N, int S, const int32_t* __restrict__ cond, const int32_t* __restrict__ uncond,
+    const float* __restrict__ s_sum, const float* __restrict__ t_sum,
+    const int32_t* __restrict__ count, float lo, float hi, int flags, float* ifd_t, float* ifd_s,
+    float* delta, uint8_t* keep, int32_t* n_keep) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  int kept = 0;
+  if (i < N) {
+    const int c = cond[i], u = uncond[i];
+    const float nan = __int_as_float(0x7fc00000);
+    float it = nan, is = nan;
+    if (c >= 0 && c < S && u >= 0 && u < S) {
+      const int nc = count[c], nu = count[u];
+      if (nc > 0 && nu > 0) {
+        const float fc = static_cast<float>(nc), fu = static_cast<float>(nu);
+        const float tu = __fdiv_rn(t_sum[u], fu), su = __fdiv_rn(s_sum[u], fu);
+        if (tu != 0.f) it = __fdiv_rn(__fdiv_rn(t_sum[c], fc), tu);
+        if (su != 0.f) is = __fdiv_rn(__fdiv_rn(s_sum[c], fc), su);
+      }
+    }
+    const float dl = __fsub_rn(it, is);
+    bool k = (dl >= lo) && (dl <= hi);  // false for NaN
+    if (flags & 1) k = k && (it <= 1.0f);
+    if (ifd_t != nullptr) ifd_t[i] = it;
+    if (ifd_s != nullptr) ifd_s[i] = is;
+    if (delta != nullptr) delta[i] = dl;
+    keep[i] = k ? 1 : 0;
+    kept = k ? 1 : 0;
+  }
+  kept = warp_sum_int(kept);
+  if ((threadIdx.x & 31) == 0 && kept != 0) atomicAdd(n_keep, kept);
+}
+
+// fp32 [T, d] accumulator -> bf16 [T, ld] output, 8 elements per thread.
+__global__ void __launch_bounds__(256) f32_to_bf16_rows_kernel(const float* __restrict__ src, int T,
+                                                              int d, __nv_bfloat16* dst,
+                                                              long long ld) {
+  const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int per_row = d / 8;
+  if (i >= static_cast<long long>(T) * per_row) return;
+  const int t = static_cast<int>(i / per_row), c = static_cast<int>(i % per_row) * 8;
+  const float4 a = *reinterpret_cast<const float4*>(src + static_cast<size_t>(t) * d + c);
+  const float4 b = *reinterpret_cast<const float4*>(src + static_cast<size_t>(t) * d + c + 4);
+  uint4 o;
+  o.x = pack_bf16x2(a.x, a.y);
+  o.y = pack_bf16x2(a.z, a.w);
+  o.z = pack_bf16x2(b.x, b.y);
+  o.w = pack_bf16x2(b.z, b.w);
+  *reinterpret_cast<uint4*>(dst + static_cast<size_t>(t) * ld + c) = o;
+}
+
+}  // namespace npd
