@@ -104,12 +104,25 @@ typedef struct npd_kd_args {
   int32_t reserved1;
   void* workspace;           /* >= npd_workspace_bytes(), 1024-byte aligned         */
   size_t workspace_bytes;
+  /* Optional timing hooks.  HOST array of n_phase_events cudaEvent_t (as void*), or NULL.
+     Event 0 is recorded on the stream before the first kernel, event i after the i-th
+     launch group, in this order: forward tiles, per-token merge, then for every
+     vocabulary chunk: gradient tiles, dW contraction, dH contraction; last the dH
+     conversion if there is one.  Groups beyond n_phase_events - 1 are not recorded.
+     npd_phase_count() tells how many groups a call has. */
+  void* const* phase_events;
+  int32_t n_phase_events;
+  int32_t reserved2;
 } npd_kd_args;
 
 /* HOST.  Bytes of workspace npd_kd_fwd_bwd needs for these arguments (pointers
  * inside args are not read).  Depends on T, d, V, grad_chunk_cols, on whether
  * gradients are requested and on the device's SM count. */
 int npd_workspace_bytes(const npd_kd_args* args, size_t* out_bytes);
+
+/* HOST.  Number of launch groups (see phase_events) npd_kd_fwd_bwd runs for these arguments,
+ * and in *out_chunks (may be NULL) the number of vocabulary chunks of the backward. */
+int npd_phase_count(const npd_kd_args* args, int32_t* out_groups, int32_t* out_chunks);
 
 /* Fused forward + backward of the distillation term (see the struct).  `args`
  * is a HOST struct holding device pointers.  Enqueues on `cuda_stream`. */

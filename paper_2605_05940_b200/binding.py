@@ -24,7 +24,7 @@ NPD_KD_ACCUMULATE_DW = 1
 NPD_SELECT_TEACHER_IFD_LE_1 = 1
 NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32, NPD_GEMM_ADD_BF16 = range(5)
 
-EXPORTS = ("npd_workspace_bytes", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
+EXPORTS = ("npd_workspace_bytes", "npd_phase_count", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
            "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16")
 
 
@@ -48,6 +48,7 @@ class npd_kd_args(C.Structure):
         ("d_weight_dtype", C.c_int32), ("flags", C.c_int32),
         ("grad_chunk_cols", C.c_int32), ("reserved1", C.c_int32),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("phase_events", C.POINTER(C.c_void_p)), ("n_phase_events", C.c_int32), ("reserved2", C.c_int32),
     ]
 
 
@@ -67,6 +68,7 @@ def lib() -> C.CDLL:
         l.npd_strerror.argtypes = [C.c_int]
         l.npd_workspace_bytes.argtypes = [C.POINTER(npd_kd_args), C.POINTER(C.c_size_t)]
         l.npd_kd_fwd_bwd.argtypes = [C.POINTER(npd_kd_args), C.c_void_p]
+        l.npd_phase_count.argtypes = [C.POINTER(npd_kd_args), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         l.npd_kd_fwd_bwd_host.argtypes = [C.POINTER(npd_kd_args), C.POINTER(npd_kd_args), C.c_void_p]
         l.npd_segment_stats.argtypes = [C.c_int32, C.c_int32] + [C.c_void_p] * 13
         l.npd_select.argtypes = ([C.c_int32] + [C.c_void_p] * 5 + [C.c_int32, C.c_float, C.c_float, C.c_int32]
@@ -129,6 +131,13 @@ def npd_workspace_bytes(args: npd_kd_args) -> int:
     out = C.c_size_t(0)
     _check(lib().npd_workspace_bytes(C.byref(args), C.byref(out)), "npd_workspace_bytes")
     return out.value
+
+
+def npd_phase_count(args: npd_kd_args):
+    """(launch groups, vocabulary chunks) of a call with these arguments."""
+    g, c = C.c_int32(0), C.c_int32(0)
+    _check(lib().npd_phase_count(C.byref(args), C.byref(g), C.byref(c)), "npd_phase_count")
+    return g.value, c.value
 
 
 def npd_kd_fwd_bwd(args: npd_kd_args, stream=None) -> None:
@@ -209,8 +218,11 @@ class KDStep:
         self.kl = torch.empty(T, **f32)
         self.nll_student = torch.empty(T, **f32)
         self.nll_teacher = torch.empty(T, **f32)
-        self.d_hidden = torch.empty((T, d), dtype=torch.bfloat16, device=dev) if grads else None
-        self.d_weight = torch.empty((V, d), dtype=dw_dtype, device=dev) if grads else None
+        # the gradients use the row strides of the tensors they belong to (ldh, ldw)
+        self.d_hidden = (torch.empty_strided((T, d), (batch.hidden.stride(0), 1), dtype=torch.bfloat16,
+                                             device=dev) if grads else None)
+        self.d_weight = (torch.empty_strided((V, d), (batch.weight.stride(0), 1), dtype=dw_dtype,
+                                             device=dev) if grads else None)
         self.grad_scale = (1.0 / max(batch.n_loss, 1)) if grad_scale is None else grad_scale
         self._kw = dict(cu_seqlens=batch.cu_seqlens, loss_mask=batch.loss_mask, labels=batch.labels,
                         temperature=batch.tau, grad_scale=self.grad_scale, kl=self.kl,
@@ -226,6 +238,27 @@ class KDStep:
 
     def run(self, stream=None):
         npd_kd_fwd_bwd(self.args, stream)
+
+    def run_with_phase_times(self, stream=None):
+        """One step with the library's phase events attached.  Returns a list of
+        (group name, milliseconds); synchronises."""
+        groups, chunks = npd_phase_count(self.args)
+        names = ["forward_tiles", "merge"]
+        for _ in range(chunks):
+            names += ["gradient_tiles", "dweight_gemm", "dhidden_gemm"]
+        names += ["dhidden_convert"] * (groups - len(names))
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(groups + 1)]
+        # an event only owns a CUDA handle once it has been recorded
+        s = torch.cuda.current_stream() if stream is None else stream
+        for e in evs:
+            e.record(s)
+        arr = (C.c_void_p * len(evs))(*[e.cuda_event for e in evs])
+        a = npd_kd_args.from_buffer_copy(self.args)
+        a.phase_events = C.cast(arr, C.POINTER(C.c_void_p))
+        a.n_phase_events = len(evs)
+        npd_kd_fwd_bwd(a, stream)
+        torch.cuda.synchronize()
+        return [(names[i], evs[i].elapsed_time(evs[i + 1])) for i in range(groups)]
 
     def status(self, stream=None) -> int:
         return npd_last_status(self._ws_view, stream)

@@ -68,7 +68,11 @@ constexpr int OFF_Z = OFF_B + STAGES * B_BYTES;
 constexpr int OFF_BAR = OFF_Z + 2 * ZQ * ZSUB_BYTES;
 constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * ZQ;
 constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;
-constexpr float kNegClamp = -1.0e30f;      // finite stand-in for -inf teacher logits
+// Teacher logits are clamped below at this value: a finite stand-in for the -inf entries of
+// a densified top-k teacher.  It is small enough that 2^((clamp - row max) * scale) is 0 for
+// any sane row, and small enough in magnitude that fp32 still resolves differences of scaled
+// logits near it (a huge stand-in would turn "x*scale - max" into a rounding-error blow-up).
+constexpr float kNegClamp = -30000.0f;
 }  // namespace kd_cfg
 
 template <int kMode, bool kTauIsOne>

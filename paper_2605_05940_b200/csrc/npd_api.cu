@@ -131,7 +131,7 @@ int check_args(const npd_kd_args* a, bool need_pointers) {
   if (a->teacher_dtype == NPD_DTYPE_F32) return NPD_EUNSUPPORTED;
   if (a->teacher_dtype != NPD_DTYPE_BF16) return NPD_EINVAL;
   if (a->d_weight_dtype != NPD_DTYPE_BF16 && a->d_weight_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
-  if (a->grad_chunk_cols < 0) return NPD_EINVAL;
+  if (a->grad_chunk_cols < 0 || a->n_phase_events < 0) return NPD_EINVAL;
   if (a->d % 64 != 0) return NPD_ESHAPE;
   if (a->ldh < a->d || a->ldw < a->d || a->ldt < a->V) return NPD_ESHAPE;
   if (a->cu_seqlens != nullptr && (a->S < 1 || a->S > a->T)) return NPD_ESHAPE;
@@ -147,6 +147,17 @@ int check_args(const npd_kd_args* a, bool need_pointers) {
   if (a->d_weight != nullptr && a->d_weight_dtype == NPD_DTYPE_F32 && (a->ldw % 4)) return NPD_EALIGN;
   return NPD_OK;
 }
+
+// Records the caller's optional phase events in order.
+struct PhaseRecorder {
+  void* const* ev;
+  int n, next;
+  cudaStream_t st;
+  void mark() {
+    if (ev != nullptr && next < n && ev[next] != nullptr) cudaEventRecord(static_cast<cudaEvent_t>(ev[next]), st);
+    ++next;
+  }
+};
 
 template <typename K>
 int set_smem(K kernel, int bytes) {
@@ -241,6 +252,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   float* lse_b = reinterpret_cast<float*>(ws + pl.off_lse_b);
   float* coef = reinterpret_cast<float*>(ws + pl.off_coef);
   if (cudaMemsetAsync(status, 0, 64, st) != cudaSuccess) return NPD_ECUDA;
+  PhaseRecorder rec{a->phase_events, a->n_phase_events, 0, st};
 
   const bool tau_one = a->temperature == 1.0f;
   const float scale2 = 1.4426950408889634f / a->temperature;
@@ -259,6 +271,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     ++g_launches;
   }
 
+  rec.mark();
   // ---- forward: statistics per (row block, vocabulary run), then the per-token merge ----
   KdTileParams kp{};
   kp.T = a->T;
@@ -273,6 +286,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   kp.partials = partials;
   kp.status = status;
   if ((rc = launch_kd_tile<kForward>(tau_one, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
+  rec.mark();
 
   CombineParams cp{};
   cp.T = a->T;
@@ -303,6 +317,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     kd_combine_kernel<false><<<(a->T + 7) / 8, 256, 0, st>>>(cp);
   ++g_launches;
   if (cudaGetLastError() != cudaSuccess) return NPD_ECUDA;
+  rec.mark();
   if (!pl.grads) return NPD_OK;
 
   // ---- backward: per vocabulary chunk, gradient tiles -> scratch -> dW rows and dH partial ----
@@ -326,6 +341,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     gp.coef = coef;
     gp.g_col0 = col0;
     if ((rc = launch_kd_tile<kGradient>(tau_one, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
+    rec.mark();
 
     // dW[col0 .. col0+cols) = G_chunk^T H       (M = vocabulary rows, N = d, K = T)
     GemmParams gw{};
@@ -343,6 +359,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
       gw.out_mode = kOutStoreBF16;
     }
     if ((rc = launch_gemm(true, true, gbuf, ldg, a->hidden, a->ldh, gw, di.sms, st)) != NPD_OK) return rc;
+    rec.mark();
 
     // dH (+)= G_chunk W[col0 .. col0+cols)      (M = T, N = d, K = vocabulary rows of the chunk)
     GemmParams gh{};
@@ -362,6 +379,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     }
     const __nv_bfloat16* wc = static_cast<const __nv_bfloat16*>(a->weight) + static_cast<size_t>(col0) * a->ldw;
     if ((rc = launch_gemm(false, true, gbuf, ldg, wc, a->ldw, gh, di.sms, st)) != NPD_OK) return rc;
+    rec.mark();
   }
   if (pl.nchunks > 1) {
     const long long n = static_cast<long long>(a->T) * (a->d / 8);
@@ -369,7 +387,25 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
         dh_acc, a->T, a->d, static_cast<__nv_bfloat16*>(a->d_hidden), a->ldh);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return NPD_ECUDA;
+    rec.mark();
   }
+  return NPD_OK;
+}
+
+int npd_phase_count(const npd_kd_args* args, int32_t* out_groups, int32_t* out_chunks) {
+  if (out_groups == nullptr) return NPD_EINVAL;
+  int rc = check_args(args, false);
+  if (rc != NPD_OK) return rc;
+  DeviceInfo di;
+  if ((rc = device_info(&di)) != NPD_OK) return rc;
+  Plan pl;
+  make_plan(args, di.sms, &pl);
+  int chunks = 0;
+  if (pl.grads)
+    for (int c = 0; c < pl.nchunks; ++c)
+      if (args->V - c * pl.chunk_cols > 0) ++chunks;
+  *out_groups = 2 + 3 * chunks + ((pl.grads && pl.nchunks > 1) ? 1 : 0);
+  if (out_chunks != nullptr) *out_chunks = chunks;
   return NPD_OK;
 }
 

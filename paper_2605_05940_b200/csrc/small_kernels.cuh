@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
   }
   if (lane == 0) {
     const float kl = kLn2 * (p.scale2 * (cr / sa) - lse_a + lse_b);
-    p.kl[t] = on ? fmaxf(kl, 0.f) : 0.f;
+    p.kl[t] = on ? (kl < 0.f ? 0.f : kl) : 0.f;  // rounding may dip below 0; NaN stays NaN
     if (p.nll_s != nullptr) p.nll_s[t] = nll_s;
     if (p.nll_t != nullptr) p.nll_t[t] = nll_t;
     p.lse2_a[t] = lse_a;

@@ -1,0 +1,122 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py
+times (library defaults), on sampled outputs the oracle computes one by one, plus
+properties that hold at any size."""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import npd_oracle as orc
+from paper_2605_05940_b200 import binding as B
+from paper_2605_05940_b200 import synth_inputs as syn
+
+from _parity import GRAD_FROB, assert_losses_close, frob, host, run_step
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _sample_rows(b, n, seed):
+    rng = np.random.default_rng(seed)
+    cu = b.cu_seqlens.cpu().numpy()
+    fixed = {0, b.T - 1, int(cu[1]) - 1, int(cu[1]), 127, 128, b.T - 129}
+    rows = sorted(fixed | set(rng.integers(0, b.T, size=n).tolist()))
+    return np.asarray([r for r in rows if 0 <= r < b.T])
+
+
+def _check_sampled_rows(b, step, rows):
+    W = host(b.weight)
+    r = torch.from_numpy(rows).to(DEV)
+    H, Z = host(b.hidden[r]), host(b.teacher[r])
+    y, m = b.labels[r].cpu().numpy(), b.loss_mask[r].cpu().numpy()
+    kl, ns, nt = orc.kd_token_losses(H, W, Z, y, m, b.tau)
+    assert_losses_close(host(step.kl[r]), kl, "kl rows")
+    assert_losses_close(host(step.nll_student[r]), ns, "nll_student rows")
+    assert_losses_close(host(step.nll_teacher[r]), nt, "nll_teacher rows")
+    dH = orc.kd_dhidden_rows(H, W, Z, m, b.tau, step.grad_scale, np.arange(len(rows)))
+    assert frob(host(step.d_hidden[r]), dH) <= GRAD_FROB
+    on = m == 1
+    assert on.any() and (~on).any()
+    assert np.all(host(step.d_hidden[r])[~on] == 0)
+    return W
+
+
+def _check_properties(b, step):
+    m = b.loss_mask.bool()
+    assert float(step.kl[~m].abs().max()) == 0.0
+    assert bool((step.kl[m] > 0).all()) and bool(torch.isfinite(step.kl).all())
+    assert float(step.d_hidden[~m].float().abs().max()) == 0.0
+    dW = step.d_weight.float()
+    colsum = dW.sum(dim=0)
+    # rows of dO_S sum to zero over the vocabulary, hence so do the columns of dW
+    assert float(colsum.norm() / dW.norm()) < 5e-2
+    # segment statistics: counts bit-exact against the definition, at any size
+    got = B.npd_segment_stats(b.cu_seqlens, b.loss_mask, b.labels, step.kl, step.nll_student,
+                              step.nll_teacher)
+    cu = b.cu_seqlens.cpu().numpy()
+    y, mm = b.labels.cpu().numpy(), b.loss_mask.cpu().numpy()
+    z = np.zeros(b.T)
+    ref_cnt = orc.segment_stats(cu, mm, y, z, z, z)[3]
+    assert np.array_equal(got[3].cpu().numpy(), ref_cnt)
+    assert np.array_equal(got[4].cpu().numpy(), orc.segment_ids(cu, b.T))
+    ref_kl = orc.segment_stats(cu, mm, y, host(step.kl), z, z)[0]      # the reduction itself
+    assert_losses_close(host(got[0]), ref_kl, "kl_sum")
+
+
+def test_config2_full_size_sampled_rows_and_dweight_rows():
+    b = syn.config2_1b(device=DEV)
+    step = run_step(b)                       # library defaults, as bench.py runs it
+    rows = _sample_rows(b, 40, 0)
+    W = _check_sampled_rows(b, step, rows)
+    _check_properties(b, step)
+    # dW rows need every token's softmax denominator: the oracle runs all T tokens
+    vr = np.asarray([0, 1, 255, 256, 4095, 4096, 77777, b.V - 129, b.V - 128, b.V - 1])
+    ref = orc.kd_dweight_rows(b.hidden.float().cpu().numpy(), W, b.teacher.float().cpu().numpy(),
+                              b.loss_mask.cpu().numpy(), b.tau, step.grad_scale, vr, token_group=512)
+    got = host(step.d_weight[torch.from_numpy(vr).to(DEV)])
+    assert frob(got, ref) <= GRAD_FROB
+
+
+def test_config3_full_size_sampled_rows_temperature_two():
+    b = syn.config3_rows(device=DEV)
+    assert (b.T, b.d, b.tau) == (32768, 2048, 2.0)
+    step = run_step(b)
+    _check_sampled_rows(b, step, _sample_rows(b, 24, 1))
+    _check_properties(b, step)
+
+
+def test_config4_full_size_segments_and_selection_sampled():
+    b = syn.config4_short(device=DEV)
+    assert b.S > 350
+    step = run_step(b)
+    _check_sampled_rows(b, step, _sample_rows(b, 24, 2))
+    _check_properties(b, step)
+    # selection on whole samples the oracle can afford: the first 12 pairs (24 segments)
+    cu = b.cu_seqlens.cpu().numpy()
+    n_pairs, t_end = 12, int(cu[24])
+    W = host(b.weight)
+    kl, ns, nt = orc.kd_token_losses(host(b.hidden[:t_end]), W, host(b.teacher[:t_end]),
+                                     b.labels[:t_end].cpu().numpy(), b.loss_mask[:t_end].cpu().numpy(), b.tau)
+    ref = orc.segment_stats(cu[:25], b.loss_mask[:t_end].cpu().numpy(), b.labels[:t_end].cpu().numpy(), kl, ns, nt)
+    got = B.npd_segment_stats(b.cu_seqlens, b.loss_mask, b.labels, step.kl, step.nll_student, step.nll_teacher)
+    for g, r in zip(got[:3], ref[:3]):
+        assert_losses_close(host(g[:24]), r, "segment sums")
+    cond, unc = np.arange(n_pairs) * 2, np.arange(n_pairs) * 2 + 1
+    d0 = orc.delta_ifd_select(cond, unc, ref[1], ref[2], ref[3], 0.0, 1.0)[2]
+    hi = orc.nearest_rank_percentile(d0, 0.8)
+    o = orc.delta_ifd_select(cond, unc, ref[1], ref[2], ref[3], 0.0, hi)
+    sel = B.npd_select(b.cond_seg[:n_pairs], b.uncond_seg[:n_pairs], got[1], got[2], got[3], 0.0, hi)
+    near = (np.abs(o[2]) <= 1e-4) | (np.abs(o[2] - hi) <= 1e-4)
+    assert np.array_equal(sel[3].cpu().numpy()[~near], o[3][~near])
+    assert_losses_close(host(sel[2]), o[2], "delta")
+
+
+def test_config5_full_size_sampled_rows():
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2**30:
+        pytest.skip("needs about 30 GB of free device memory")
+    b = syn.config5_large(device=DEV)
+    assert (b.T, b.d) == (65536, 4096)
+    step = run_step(b)
+    _check_sampled_rows(b, step, _sample_rows(b, 16, 3))
+    _check_properties(b, step)

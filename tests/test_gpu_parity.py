@@ -1,0 +1,272 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the CPU oracle
+on the same seeded inputs, element by element, at sizes the oracle finishes in
+seconds that still span several tiles and ragged tails; plus the edge cases."""
+
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import npd_oracle as orc
+from paper_2605_05940_b200 import binding as B
+from paper_2605_05940_b200 import synth_inputs as syn
+
+from _parity import (GRAD_FROB, assert_losses_close, check_full_parity, check_stats_and_select, frob,
+                     host, oracle_inputs, run_step)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+# ----------------------------------------------------------------------------------------------
+# the tensor-core contraction building block (dH = dO W, dW = dO^T H)
+# ----------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("a_mn,b_mn", [(False, False), (True, False), (False, True), (True, True)])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (296, 520, 200), (8, 8, 8), (1000, 264, 4200)])
+def test_gemm_operand_layouts(a_mn, b_mn, M, N, K):
+    g = torch.Generator(device=DEV).manual_seed(M * 7 + N * 3 + K)
+    A = torch.randn((K, M) if a_mn else (M, K), device=DEV, generator=g).to(torch.bfloat16)
+    Bm = torch.randn((K, N) if b_mn else (N, K), device=DEV, generator=g).to(torch.bfloat16)
+    out = torch.full((M, N), float("nan"), device=DEV)
+    B.npd_gemm_bf16(A, Bm, out, a_mn_major=a_mn, b_mn_major=b_mn)
+    torch.cuda.synchronize()
+    Ah, Bh = host(A), host(Bm)
+    ref = orc.student_logits(Ah.T if a_mn else Ah, Bh.T if b_mn else Bh)   # A B^T in fp64
+    assert frob(host(out), ref) < 2e-5      # fp32 accumulation over K
+
+
+def test_gemm_output_modes_and_split_k():
+    g = torch.Generator(device=DEV).manual_seed(5)
+    M, N, K = 520, 776, 1800
+    A = torch.randn((M, K), device=DEV, generator=g).to(torch.bfloat16)
+    Bm = torch.randn((K, N), device=DEV, generator=g).to(torch.bfloat16)
+    ref = orc.student_logits(host(A), host(Bm).T)
+    base = torch.randn((M, N), device=DEV, generator=g)
+    out = base.clone()
+    B.npd_gemm_bf16(A, Bm, out, b_mn_major=True, out_mode=B.NPD_GEMM_ADD_F32)
+    assert frob(host(out), ref + host(base)) < 2e-5
+    out = base.clone()
+    B.npd_gemm_bf16(A, Bm, out, b_mn_major=True, out_mode=B.NPD_GEMM_ATOMIC_F32, k_splits=5)
+    assert frob(host(out), ref + host(base)) < 2e-5
+    outb = torch.empty((M, N), device=DEV, dtype=torch.bfloat16)
+    B.npd_gemm_bf16(A, Bm, outb, b_mn_major=True, out_mode=B.NPD_GEMM_STORE_BF16)
+    assert frob(host(outb), ref) < 4e-3
+    # strided output and operands
+    big = torch.zeros((M, N + 24), device=DEV)
+    Apad = torch.zeros((M, K + 8), device=DEV, dtype=torch.bfloat16)
+    Apad[:, :K] = A
+    B.npd_gemm_bf16(Apad[:, :K], Bm, big[:, :N], b_mn_major=True)
+    torch.cuda.synchronize()
+    assert frob(host(big[:, :N]), ref) < 2e-5 and float(big[:, N:].abs().max()) == 0.0
+
+
+# ----------------------------------------------------------------------------------------------
+# the fused step
+# ----------------------------------------------------------------------------------------------
+def test_config1_tiny_all_outputs():
+    b = syn.config1_tiny(device=DEV, teacher_dtype=torch.bfloat16)
+    step = run_step(b, dw_dtype=torch.float32)
+    kl, ns, nt = check_full_parity(b, step)
+    check_stats_and_select(b, step, kl, ns, nt)
+    assert np.array_equal(b.cu_seqlens.cpu().numpy(), [0, 32, 96, 192, 256])
+
+
+@pytest.mark.parametrize("chunk", [0, 256, 1024])
+def test_scaled_config2_multi_tile_ragged(chunk):
+    # 6 row blocks with a ragged last one, 12 vocabulary tiles with a ragged tail, 2 k-steps
+    b = syn.scaled("c2", device=DEV, T=700, d=128, V=3000, min_len=20, max_len=300)
+    step = run_step(b, grad_chunk_cols=chunk)
+    kl, ns, nt = check_full_parity(b, step)
+    check_stats_and_select(b, step, kl, ns, nt)
+
+
+def test_scaled_config3_temperature_two_and_row_boundaries():
+    b = syn.scaled("c3", device=DEV, rows=2, row_len=512, d=192, V=5000)
+    assert b.tau == 2.0
+    step = run_step(b, grad_chunk_cols=2048, dw_dtype=torch.float32)
+    kl, ns, nt = check_full_parity(b, step)
+    check_stats_and_select(b, step, kl, ns, nt)
+
+
+def test_scaled_config5_wide_hidden():
+    b = syn.scaled("c5", device=DEV, T=1100, d=1024, V=2304)
+    step = run_step(b, grad_chunk_cols=768)
+    check_full_parity(b, step)
+
+
+def test_config4_short_segments_full_segment_count_and_selection():
+    # all ~400 paired segments of the workload, vocabulary and width reduced for the oracle
+    b = syn.scaled("c4", device=DEV, T=16384, d=128, V=2048)
+    assert b.S > 350
+    step = run_step(b, grads=False)
+    kl, ns, nt = check_full_parity(b, step, check_grads=False)
+    frac = check_stats_and_select(b, step, kl, ns, nt, q=0.8)
+    assert 0.2 < frac < 0.9       # the 80th-percentile threshold keeps a real subset
+
+
+def test_runs_are_bitwise_reproducible():
+    b = syn.scaled("c2", device=DEV, T=700, d=128, V=3000, min_len=20, max_len=300)
+    s1 = run_step(b, grad_chunk_cols=1024)
+    outs1 = [t.clone() for t in (s1.kl, s1.nll_student, s1.nll_teacher, s1.d_hidden, s1.d_weight)]
+    s1.run()
+    torch.cuda.synchronize()
+    for a, c in zip(outs1, (s1.kl, s1.nll_student, s1.nll_teacher, s1.d_hidden, s1.d_weight)):
+        assert torch.equal(a, c)
+
+
+# ----------------------------------------------------------------------------------------------
+# edge cases
+# ----------------------------------------------------------------------------------------------
+def _mini(T=40, d=64, V=96, seed=3, **kw):
+    return syn.scaled("c2", device=DEV, T=T, d=d, V=V, seed_base=seed, min_len=kw.pop("min_len", 5),
+                      max_len=kw.pop("max_len", 17))
+
+
+def test_single_token_single_segment_and_tiny_vocab():
+    b = _mini(T=1, V=8, min_len=1, max_len=1)
+    b.loss_mask[:] = 1
+    b.labels[:] = 3
+    step = run_step(b)
+    check_full_parity(b, step)
+    got = B.npd_segment_stats(b.cu_seqlens, b.loss_mask, b.labels, step.kl, step.nll_student, step.nll_teacher)
+    assert got[3].tolist() == [1] and got[4].tolist() == [0]
+
+
+def test_all_tokens_masked_gives_zero_loss_and_zero_gradients():
+    b = _mini()
+    b.loss_mask[:] = 0
+    step = run_step(b, dw_dtype=torch.float32)
+    assert float(step.kl.abs().max()) == 0 and float(step.nll_student.abs().max()) == 0
+    assert float(step.d_hidden.float().abs().max()) == 0 and float(step.d_weight.abs().max()) == 0
+
+
+def test_optional_inputs_may_be_null():
+    b = _mini()
+    H, W, Z, y, m = oracle_inputs(b)
+    T = b.T
+    kl = torch.empty(T, device=DEV)
+    a = B.make_kd_args(b.hidden, b.weight, b.teacher, kl=kl, temperature=1.0, grad_scale=1.0)
+    ws = torch.empty(B.npd_workspace_bytes(a) + 1024, dtype=torch.uint8, device=DEV)
+    off = (-ws.data_ptr()) % 1024
+    a = B.make_kd_args(b.hidden, b.weight, b.teacher, kl=kl, temperature=1.0, grad_scale=1.0,
+                       workspace=ws[off:])
+    B.npd_kd_fwd_bwd(a)
+    torch.cuda.synchronize()
+    ref, _, _ = orc.kd_token_losses(H, W, Z, np.full(T, -1), np.ones(T), 1.0)
+    assert_losses_close(host(kl), ref, "kl without mask/labels/cu_seqlens")
+
+
+def test_padded_strides_and_teacher_columns_beyond_vocab():
+    b = _mini(T=150, d=64, V=1001 - 1)          # V = 1000
+    V, T, d = b.V, b.T, b.d
+    zpad = torch.full((T, V + 24), 77.0, device=DEV, dtype=torch.bfloat16)   # junk beyond V
+    zpad[:, :V] = b.teacher
+    hpad = torch.zeros((T, d + 8), device=DEV, dtype=torch.bfloat16)
+    hpad[:, :d] = b.hidden
+    b2 = syn.KDBatch(b.name, T, d, V, b.S, hpad[:, :d], b.weight, zpad[:, :V], b.cu_seqlens,
+                     b.loss_mask, b.labels, b.tau)
+    step = B.KDStep(b2)
+    assert step.args.ldh == d + 8 and step.args.ldt == V + 24 and step.d_hidden.stride(0) == d + 8
+    step.run()
+    torch.cuda.synchronize()
+    check_full_parity(b, step)
+
+
+def test_minus_inf_teacher_entries_dense_top_k():
+    # a top-k teacher densified with -inf outside its support (Eq. 2 on the top-k support)
+    b = _mini(T=70, V=600)
+    z = b.teacher.float()
+    kth = z.topk(10, dim=1).values[:, -1:]
+    b.teacher = torch.where(z >= kth, z, torch.full_like(z, float("-inf"))).to(torch.bfloat16)
+    step = run_step(b, dw_dtype=torch.float32)
+    assert torch.isfinite(step.kl).all() and torch.isfinite(step.d_weight).all()
+    check_full_parity(b, step)
+
+
+def test_forward_only_and_f32_accumulating_dweight():
+    b = _mini(T=200, V=520)
+    f = run_step(b, grads=False)
+    g = run_step(b, dw_dtype=torch.float32)
+    assert torch.equal(f.kl, g.kl) and f.d_hidden is None
+    first = g.d_weight.clone()
+    g.args.flags = B.NPD_KD_ACCUMULATE_DW
+    g.run()
+    torch.cuda.synchronize()
+    assert frob(host(g.d_weight), 2 * host(first)) < 1e-6
+
+
+def test_malformed_cu_seqlens_is_reported_not_faulted():
+    b = _mini(T=60)
+    good = b.cu_seqlens.clone()
+    for bad in ([0, 70, 60], [1] + good.tolist()[1:], good.tolist()[:-1] + [59],
+                [0, 30, 30, 60], [0, 40, 20, 60], [0, -5, 60]):
+        b.cu_seqlens = torch.tensor(bad, dtype=torch.int32, device=DEV)
+        b.S = len(bad) - 1
+        step = B.KDStep(b, grads=False)
+        step.run()
+        assert step.status() == B.NPD_ESEQ, bad
+        st = torch.zeros(1, dtype=torch.int32, device=DEV)
+        B.npd_segment_stats(b.cu_seqlens, b.loss_mask, b.labels, step.kl, step.nll_student,
+                            step.nll_teacher, status=st)
+        assert int(st.item()) == B.NPD_ESEQ
+    b.cu_seqlens, b.S = good, good.numel() - 1
+    step = B.KDStep(b, grads=False)
+    step.run()
+    assert step.status() == B.NPD_OK
+
+
+def test_workspace_and_option_errors():
+    b = _mini()
+    step = B.KDStep(b)
+    a = B.npd_kd_args.from_buffer_copy(step.args)
+    a.workspace_bytes = step.args.workspace_bytes - 1
+    assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EWORKSPACE
+    a = B.npd_kd_args.from_buffer_copy(step.args)
+    a.workspace = step.args.workspace + 16
+    assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EWORKSPACE
+    a = B.npd_kd_args.from_buffer_copy(step.args)
+    a.teacher_dtype = B.NPD_DTYPE_F32
+    assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EUNSUPPORTED
+
+
+def test_select_matches_float32_oracle_bit_for_bit():
+    rng = np.random.default_rng(0)
+    S = 4001
+    N = 2000
+    count = rng.integers(0, 40, size=S).astype(np.int32)
+    s_sum = (rng.random(S) * 30).astype(np.float32)
+    t_sum = (rng.random(S) * 30).astype(np.float32)
+    s_sum[5] = 0.0
+    cond = rng.integers(0, S, size=N).astype(np.int32)
+    unc = rng.integers(0, S, size=N).astype(np.int32)
+    to = lambda x: torch.from_numpy(x).to(DEV)
+    for flags in (0, B.NPD_SELECT_TEACHER_IFD_LE_1):
+        it, is_, dl, keep, n = B.npd_select(to(cond), to(unc), to(s_sum), to(t_sum), to(count), 0.0, 0.8, flags)
+        o = orc.delta_ifd_select(cond, unc, s_sum, t_sum, count, 0.0, 0.8,
+                                 require_teacher_ifd_le_1=bool(flags), dtype=np.float32)
+        assert np.array_equal(it.cpu().numpy(), o[0], equal_nan=True)
+        assert np.array_equal(is_.cpu().numpy(), o[1], equal_nan=True)
+        assert np.array_equal(dl.cpu().numpy(), o[2], equal_nan=True)
+        assert np.array_equal(keep.cpu().numpy(), o[3]) and int(n.item()) == o[4]
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    b = syn.scaled("c2", device=DEV, T=300, d=64, V=520, min_len=20, max_len=90)
+    ref = run_step(b)
+    pin = lambda t: t.cpu().pin_memory()
+    hh, hz, hcu, hm, hy = map(pin, (b.hidden, b.teacher, b.cu_seqlens, b.loss_mask, b.labels))
+    hkl, hns, hnt = (torch.empty(b.T).pin_memory() for _ in range(3))
+    # fresh device staging buffers (zeroed), resident weight
+    stage = syn.KDBatch(b.name, b.T, b.d, b.V, b.S, torch.zeros_like(b.hidden), b.weight,
+                        torch.zeros_like(b.teacher), torch.zeros_like(b.cu_seqlens),
+                        torch.zeros_like(b.loss_mask), torch.zeros_like(b.labels), b.tau)
+    step = B.KDStep(stage, grad_scale=ref.grad_scale)
+    hargs = B.make_kd_args(hh, b.weight, hz, cu_seqlens=hcu, loss_mask=hm, labels=hy, kl=hkl,
+                           nll_student=hns, nll_teacher=hnt, temperature=b.tau)
+    B.npd_kd_fwd_bwd_host(hargs, step.args)
+    torch.cuda.synchronize()
+    assert step.status() == B.NPD_OK
+    assert torch.equal(hkl, ref.kl.cpu()) and torch.equal(hns, ref.nll_student.cpu())
+    assert torch.equal(hnt, ref.nll_teacher.cpu())
+    assert torch.equal(step.d_hidden, ref.d_hidden) and torch.equal(step.d_weight, ref.d_weight)
