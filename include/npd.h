@@ -192,6 +192,40 @@ const char* npd_strerror(int status);
  * enqueued (for launch accounting in benchmarks). */
 int npd_last_launch_count(void);
 
+/*
+ * Forward pass without any workspace from the caller.  (The paper has no counterpart
+ * to this entry point; it exists for deployment.)
+ *
+ * For callers that cannot allocate device memory: code running inside a host framework
+ * that took the whole device memory for its own pool at start-up, so that a fresh
+ * cudaMalloc fails, and steady-state loops that may not stall the device, which
+ * cudaMalloc and cudaFree do.  The scratch of the forward pass (softmax partials per
+ * vocabulary split, per-token log-sum-exps, status word) lives in a fixed array inside
+ * the library image instead: NPD_STATIC_SCRATCH_BYTES (+1 KiB) on every GPU that loads
+ * the library, held until the process exits.
+ *
+ * `args` as for npd_kd_fwd_bwd, forward only: d_hidden and d_weight must be NULL
+ * (NPD_EINVAL otherwise); workspace / workspace_bytes are ignored.  The caller still
+ * passes all inputs and the kl / nll_* outputs.  A problem whose scratch
+ * (npd_workspace_bytes of the same forward-only arguments) exceeds
+ * NPD_STATIC_SCRATCH_BYTES is refused with NPD_EWORKSPACE before anything is launched;
+ * c2's forward (T=8192, V=151,936) needs about 17 MB.  The call makes no cudaMalloc,
+ * cudaFree or other allocating call.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current) and caches it; make that first call outside any stream capture.  All calls on
+ * a device share the one array and it keeps the previous call's contents: the library
+ * clears the status word at the start of every call and overwrites every partial before
+ * reading it, but two calls whose kernels overlap on the GPU (different streams, or
+ * different host threads) race on it - serialise them.
+ *
+ * host_status (HOST, may be NULL): if given, the call synchronises `cuda_stream` and
+ * stores the device-side status (NPD_OK, NPD_ESEQ, NPD_ETIMEOUT) there, as
+ * npd_last_status would; if NULL the call only enqueues.
+ */
+#define NPD_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+int npd_kd_forward_noalloc(const npd_kd_args* args, void* cuda_stream, int32_t* host_status);
+
 /* out_mode of npd_gemm_bf16 */
 enum {
   NPD_GEMM_STORE_F32 = 0,  /* D = acc                       */

@@ -25,7 +25,9 @@ NPD_SELECT_TEACHER_IFD_LE_1 = 1
 NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32, NPD_GEMM_ADD_BF16 = range(5)
 
 EXPORTS = ("npd_workspace_bytes", "npd_phase_count", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
-           "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16")
+           "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16",
+           "npd_kd_forward_noalloc")
+NPD_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 
 class NpdError(RuntimeError):
@@ -75,6 +77,7 @@ def lib() -> C.CDLL:
                                  + [C.c_void_p] * 6)
         l.npd_last_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
         l.npd_last_launch_count.argtypes = []
+        l.npd_kd_forward_noalloc.argtypes = [C.POINTER(npd_kd_args), C.c_void_p, C.POINTER(C.c_int32)]
         l.npd_gemm_bf16.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int32,
                                     C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64,
                                     C.c_int32, C.c_int32, C.c_void_p]
@@ -146,6 +149,16 @@ def npd_kd_fwd_bwd(args: npd_kd_args, stream=None) -> None:
 
 def npd_kd_fwd_bwd_host(host: npd_kd_args, dev: npd_kd_args, stream=None) -> None:
     _check(lib().npd_kd_fwd_bwd_host(C.byref(host), C.byref(dev), _stream(stream)), "npd_kd_fwd_bwd_host")
+
+
+def npd_kd_forward_noalloc(args: npd_kd_args, stream=None, want_status: bool = False):
+    """Forward pass on the library's built-in scratch array (no workspace, no allocation).
+    For callers that cannot allocate device memory; see include/npd.h for the limits.
+    With want_status the call synchronises the stream and returns the device status."""
+    st = C.c_int32(0)
+    _check(lib().npd_kd_forward_noalloc(C.byref(args), _stream(stream), C.byref(st) if want_status else None),
+           "npd_kd_forward_noalloc")
+    return st.value if want_status else None
 
 
 def npd_last_status(workspace: torch.Tensor, stream=None) -> int:

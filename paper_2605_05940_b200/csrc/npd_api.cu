@@ -11,6 +11,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 
 #include "gemm_sm100.cuh"
 #include "kd_tile_sm100.cuh"
@@ -481,6 +482,65 @@ int npd_last_status(const void* workspace, void* cuda_stream, int32_t* host_stat
   if (cudaMemcpyAsync(host_status, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return NPD_ECUDA;
   return cudaStreamSynchronize(st) == cudaSuccess ? NPD_OK : NPD_ECUDA;
+}
+
+// ---------------------------------------------------------------------------------------
+// Forward pass for callers that cannot allocate device memory.
+//
+// Some users of this library cannot hand it a workspace: a plug-in running inside a host
+// framework that claimed the whole device memory for its own pool at start-up (a fresh
+// cudaMalloc there simply fails), or a steady-state serving/training loop that may not
+// stall the device (cudaMalloc and cudaFree synchronise it).  For them the forward pass'
+// scratch (the per-split softmax partials, the log-sum-exps and the status word) lives
+// in the fixed array below, which is part of the library image: every GPU that loads the
+// library carries these NPD_STATIC_SCRATCH_BYTES (+1 KiB) until the process exits.
+//
+// g_static_scratch names the array for DEVICE code.  In host code the same identifier is
+// only a host-side handle, not a device address, so the real address is asked for once
+// per device with cudaGetSymbolAddress (with that device current) and cached.
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[NPD_STATIC_SCRATCH_BYTES + 1024];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};
+std::mutex g_static_scratch_mutex;
+
+// Device address of the static scratch on the current device, 1024-byte aligned.
+int static_scratch_base(uint8_t** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return NPD_ECUDA;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return NPD_ECUDA;
+    g_static_scratch_addr[dev] = ptr;
+  }
+  const uintptr_t a = reinterpret_cast<uintptr_t>(g_static_scratch_addr[dev]);
+  *out = reinterpret_cast<uint8_t*>((a + 1023) & ~static_cast<uintptr_t>(1023));
+  return NPD_OK;
+}
+}  // namespace
+
+int npd_kd_forward_noalloc(const npd_kd_args* args, void* cuda_stream, int32_t* host_status) {
+  if (args == nullptr || args->size != sizeof(npd_kd_args)) return NPD_EINVAL;
+  if (args->d_hidden != nullptr || args->d_weight != nullptr) return NPD_EINVAL;  // forward only
+  npd_kd_args a = *args;
+  a.workspace = nullptr;
+  a.workspace_bytes = 0;
+  size_t need = 0;
+  int rc = npd_workspace_bytes(&a, &need);
+  if (rc != NPD_OK) return rc;
+  if (need > static_cast<size_t>(NPD_STATIC_SCRATCH_BYTES)) return NPD_EWORKSPACE;  // problem too large
+  uint8_t* base = nullptr;
+  if ((rc = static_scratch_base(&base)) != NPD_OK) return rc;
+  a.workspace = base;
+  a.workspace_bytes = NPD_STATIC_SCRATCH_BYTES;
+  // npd_kd_fwd_bwd clears the status word itself and overwrites every partial it later reads,
+  // so nothing of the previous call's contents survives into this one.
+  if ((rc = npd_kd_fwd_bwd(&a, cuda_stream)) != NPD_OK) return rc;
+  if (host_status != nullptr) return npd_last_status(base, cuda_stream, host_status);
+  return NPD_OK;
 }
 
 int npd_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32_t a_mn_major,
