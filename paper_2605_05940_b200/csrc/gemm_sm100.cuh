@@ -8,9 +8,12 @@
 // (memory [K][rows contiguous]); the second form lets the logit-gradient block
 // and the hidden states be read as they lie in memory, with no transposes.
 //
-// One CTA per SM, 192 threads: warp 0 = TMA producer, warp 1 = MMA issuer and
-// TMEM owner, warps 2-5 = epilogue (one accumulator row per thread).  Tiles are
-// 128 x 256 x 64 with a 4-stage operand ring and a double-buffered accumulator
+// Two CTAs on neighbouring SMs (a cluster of 2) work as a pair on a 256 x 256 output tile
+// with tcgen05 .cta_group::2: each CTA stages its own 128 rows of A and its own 128 of the
+// tile's 256 rows of B (32 KB per k-step per SM) and receives its own 128 output rows in
+// tensor memory.  One CTA per SM, 192 threads: warp 0 = TMA producer, warp 1 = TMEM owner
+// and, in the leader CTA (cluster rank 0), the MMA issuer of the pair, warps 2-5 = epilogue
+// (one accumulator row per thread).  6-stage operand ring, double-buffered accumulator
 // (2 x 256 TMEM columns), so the epilogue of one tile overlaps the MMAs of the next.
 #pragma once
 
@@ -36,16 +39,18 @@ struct GemmParams {
 };
 
 namespace gemm_cfg {
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UK = 16;
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 6, UK = 16;  // BM = rows per CTA (256 per pair)
+constexpr int PM = 2 * BM;            // rows of a pair tile
+constexpr int BNH = BN / 2;           // B rows each CTA of the pair stages
 constexpr int A_BYTES = BM * BK * 2;  // 16 KB
-constexpr int B_BYTES = BN * BK * 2;  // 32 KB
+constexpr int B_BYTES = BNH * BK * 2; // 16 KB
 constexpr int THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024;  // + barriers + alignment
 }  // namespace gemm_cfg
 
 template <bool kAMn, bool kBMn>
-__global__ void __launch_bounds__(gemm_cfg::THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(gemm_cfg::THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                  const GemmParams p) {
   using namespace gemm_cfg;
@@ -61,6 +66,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();  // 0 = leader of the pair
+  const int cluster_id = blockIdx.x >> 1;
+  const int num_clusters = gridDim.x >> 1;
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
   const uint32_t tfull0 = smem_u32(bars + 2 * STAGES), tempty0 = smem_u32(bars + 2 * STAGES + 2);
 
@@ -71,20 +79,23 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull0 + 8 * b, 1);
-      mbar_init(tempty0 + 8 * b, 4);
+      mbar_init(tempty0 + 8 * b, 8);  // 4 epilogue warps of each CTA, counted in the leader
     }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmap_a);
     prefetch_tmap(&tmap_b);
   }
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
   tc_fence_before_sync();
   __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised before anything is sent to them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  const uint32_t full_leader = mapa_shared(full0, 0);
+  const uint32_t tempty_leader = mapa_shared(tempty0, 0);
 
-  const int tiles_m = (p.M + BM - 1) / BM;
+  const int tiles_m = (p.M + PM - 1) / PM;
   const int tiles_n = (p.N + BN - 1) / BN;
   const int ktiles = (p.K + BK - 1) / BK;
   const int units = tiles_m * tiles_n * p.k_splits;
@@ -94,47 +105,49 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-        const int n0 = (u % tiles_n) * BN;
-        const int m0 = ((u / tiles_n) % tiles_m) * BM;
+      for (int u = cluster_id; u < units && ok; u += num_clusters) {
+        const int n0 = (u % tiles_n) * BN + static_cast<int>(rank) * BNH;        // this CTA's B rows
+        const int m0 = ((u / tiles_n) % tiles_m) * PM + static_cast<int>(rank) * BM;  // and A rows
         const int ks = u / (tiles_n * tiles_m);
         const int kt0 = static_cast<int>(static_cast<long long>(ktiles) * ks / p.k_splits);
         const int kt1 = static_cast<int>(static_cast<long long>(ktiles) * (ks + 1) / p.k_splits);
         for (int kt = kt0; kt < kt1; ++kt, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
           if (!(ok = mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag))) break;
-          const uint32_t fb = full0 + 8 * s;
-          mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
+          // the leader's barrier counts the bytes of both CTAs' loads of this stage
+          if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * s, 2 * (A_BYTES + B_BYTES));
+          const uint32_t fb = full_leader + 8 * s;
           const uint32_t sa = smem_u32(smem_a + s * A_BYTES), sb = smem_u32(smem_b + s * B_BYTES);
           const int k0 = kt * BK;
           if (kAMn) {
 #pragma unroll
-            for (int i = 0; i < BM / 64; ++i) tma_load_2d(sa + i * 8192, &tmap_a, fb, m0 + 64 * i, k0);
+            for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(sa + i * 8192, &tmap_a, fb, m0 + 64 * i, k0);
           } else {
-            tma_load_2d(sa, &tmap_a, fb, k0, m0);
+            tma_load_2d_pair(sa, &tmap_a, fb, k0, m0);
           }
           if (kBMn) {
 #pragma unroll
-            for (int i = 0; i < BN / 64; ++i) tma_load_2d(sb + i * 8192, &tmap_b, fb, n0 + 64 * i, k0);
+            for (int i = 0; i < BNH / 64; ++i) tma_load_2d_pair(sb + i * 8192, &tmap_b, fb, n0 + 64 * i, k0);
           } else {
-            tma_load_2d(sb, &tmap_b, fb, k0, n0);
+            tma_load_2d_pair(sb, &tmap_b, fb, k0, n0);
           }
         }
       }
-      // Drain: every load issued above must have landed before the CTA may exit.
+      // Drain: a stage is released only after its loads landed and the MMAs that read it
+      // finished, so waiting for the release of the last stages covers both.
       const uint32_t last = it < STAGES ? it : STAGES;
       for (uint32_t j = 0; j < last; ++j) {
         const uint32_t i2 = it - 1 - j;
-        mbar_wait(full0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1, abort_flag);
+        mbar_wait(empty0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1, abort_flag);
       }
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, kAMn, kBMn);
+    if (rank == 0 && lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(PM, BN, kAMn, kBMn);
       uint32_t it = 0, tile = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++tile) {
+      for (int u = cluster_id; u < units && ok; u += num_clusters, ++tile) {
         const int ks = u / (tiles_n * tiles_m);
         const int kt0 = static_cast<int>(static_cast<long long>(ktiles) * ks / p.k_splits);
         const int kt1 = static_cast<int>(static_cast<long long>(ktiles) * (ks + 1) / p.k_splits);
@@ -153,11 +166,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                                      : umma_desc_sw128(sa + k * (UK * 2), 16, 1024);
             const uint64_t db = kBMn ? umma_desc_sw128(sb + k * (UK * 128), BK * 128, 1024)
                                      : umma_desc_sw128(sb + k * (UK * 2), 16, 1024);
-            umma_bf16(d_tmem, da, db, idesc, (kt > kt0 || k > 0) ? 1u : 0u);
+            umma_bf16_pair(d_tmem, da, db, idesc, (kt > kt0 || k > 0) ? 1u : 0u);
           }
-          umma_commit(empty0 + 8 * s);
+          umma_commit_pair(empty0 + 8 * s);
         }
-        if (ok) umma_commit(tfull0 + 8 * buf);
+        if (ok) umma_commit_pair(tfull0 + 8 * buf);
       }
     }
   } else {
@@ -165,9 +178,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const int lg = warp & 3;  // TMEM lane group this warp may read
     uint32_t tile = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++tile) {
+    for (int u = cluster_id; u < units && ok; u += num_clusters, ++tile) {
       const int n0 = (u % tiles_n) * BN;
-      const int m0 = ((u / tiles_n) % tiles_m) * BM;
+      const int m0 = ((u / tiles_n) % tiles_m) * PM + static_cast<int>(rank) * BM;
       const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
       if (!(ok = mbar_wait(tfull0 + 8 * buf, tph, abort_flag))) break;
       tc_fence_after_sync();
@@ -248,15 +261,18 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
       }
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty0 + 8 * buf);
+      if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);
     }
   }
 
   // ------------------------------ teardown ------------------------------------
+  // Neither CTA may leave (or free tensor memory) while its peer can still send it barrier
+  // arrivals or have MMAs reading its shared memory.
   tc_fence_before_sync();
   __syncthreads();
+  cluster_sync_all();
   tc_fence_after_sync();
-  if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+  if (warp == 1) tmem_dealloc_pair(tmem_base, TMEM_COLS);
   if (threadIdx.x == 0 && *abort_flag != 0 && p.status != nullptr) atomicCAS(p.status, 0, kStatusTimeout);
 }
 

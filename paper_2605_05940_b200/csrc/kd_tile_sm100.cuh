@@ -15,10 +15,19 @@
 //              Eq. 2), rounded to bf16 and stored to a scratch block that the two
 //              backward contractions read.
 //
+// Two CTAs on neighbouring SMs (a cluster of 2) work as a pair on a 256-token x 256-column
+// tile with tcgen05 .cta_group::2: each CTA stages its own 128 token rows of H and its own
+// 128 of the tile's 256 weight rows, so a k-step costs each SM 32 KB of operand traffic
+// instead of the 48 KB a lone 128 x 256 tile needs, and each CTA's tensor memory receives
+// the logits of its own 128 tokens for all 256 columns.
+//
 // CTA = 384 threads, one CTA per SM, persistent over work units:
-//   warp 0      TMA producer for the H and W operand stages (3-stage ring)
-//   warp 1      tcgen05.mma issuer; owns the 512 TMEM columns (2 accumulators 128x256)
-//   warp 2      TMA producer for the teacher sub-tiles (two 2-stage rings)
+//   warp 0      TMA producer for this CTA's H and W operand stages (5-stage ring); the
+//               completion of both CTAs' loads is counted on the leader's "full" barrier
+//   warp 1      leader CTA (cluster rank 0) only: tcgen05.mma issuer for the pair; commits
+//               are multicast so that "stage free" and "accumulator ready" reach both CTAs.
+//               In both CTAs this warp owns the 512 TMEM columns (2 accumulators 128x256).
+//   warp 2      TMA producer for this CTA's teacher sub-tiles (two 2-stage rings)
 //   warps 4-11  epilogue; warp w reads TMEM lanes 32*(w%4).., columns 128*((w-4)/4)..
 //               so every thread owns one token row and half of the tile's columns.
 // All exponentials are taken in base 2 on logits pre-scaled by log2(e)/tau.
@@ -37,9 +46,10 @@ struct KdTileParams {
   int T, V;
   int ksteps;       // d / 64
   int row_blocks;   // ceil(T / 128)
+  int row_pairs;    // ceil(T / 256): one pair of CTAs owns 256 token rows
   int vt_begin;     // first 256-wide vocabulary tile of this launch
   int vt_count;     // number of vocabulary tiles of this launch
-  int nsplit;       // the vt_count tiles are cut into nsplit runs; a unit = (row block, run)
+  int nsplit;       // the vt_count tiles are cut into nsplit runs; a unit = (row pair, run)
   float scale2;     // log2(e) / tau
   float tau;
   // forward
@@ -53,10 +63,11 @@ struct KdTileParams {
 };
 
 namespace kd_cfg {
-constexpr int BM = 128, BN = 256, BK = 64, UK = 16;
-constexpr int STAGES = 3;
+constexpr int BM = 128, BN = 256, BK = 64, UK = 16;  // BM = token rows per CTA (256 per pair)
+constexpr int BNH = BN / 2;                // weight rows each CTA of the pair stages
+constexpr int STAGES = 5;
 constexpr int A_BYTES = BM * BK * 2;       // 16 KB
-constexpr int B_BYTES = BN * BK * 2;       // 32 KB
+constexpr int B_BYTES = BNH * BK * 2;      // 16 KB
 constexpr int ZSUB_COLS = 64;              // teacher sub-tile: 128 rows x 64 bf16 (128 B rows)
 constexpr int ZSUB_BYTES = BM * ZSUB_COLS * 2;  // 16 KB
 constexpr int ZQ = 2;                      // ring depth per column half
@@ -76,7 +87,7 @@ constexpr float kNegClamp = -30000.0f;
 }  // namespace kd_cfg
 
 template <int kMode, bool kTauIsOne>
-__global__ void __launch_bounds__(kd_cfg::THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kd_cfg::THREADS, 1)
 kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                const __grid_constant__ CUtensorMap tmap_t, const __grid_constant__ CUtensorMap tmap_g,
                const KdTileParams p) {
@@ -90,6 +101,9 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();   // 0 = leader of the pair
+  const int cluster_id = blockIdx.x >> 1;
+  const int num_clusters = gridDim.x >> 1;
   const uint32_t full0 = smem_u32(bars);
   const uint32_t empty0 = full0 + 8 * STAGES;
   const uint32_t tfull0 = empty0 + 8 * STAGES;
@@ -104,7 +118,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(tfull0 + 8 * b, 1);
-      mbar_init(tempty0 + 8 * b, 8);
+      mbar_init(tempty0 + 8 * b, 16);  // 8 epilogue warps of each CTA, counted in the leader
     }
     for (int i = 0; i < 2 * ZQ; ++i) {
       mbar_init(zfull0 + 8 * i, 1);
@@ -117,16 +131,20 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     prefetch_tmap(&tmap_t);
     if (kMode == kGradient) prefetch_tmap(&tmap_g);
   }
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), TMEM_COLS);
+  if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
   tc_fence_before_sync();
   __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised before anything is sent to them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  const uint32_t full_leader = mapa_shared(full0, 0);
+  const uint32_t tempty_leader = mapa_shared(tempty0, 0);
 
-  const int units = p.row_blocks * p.nsplit;
+  const int units = p.row_pairs * p.nsplit;
+  // r = this CTA's 128-row block of the unit's row pair
   auto run_of = [&](int u, int& r, int& s, int& vt0, int& vt1) {
-    r = u % p.row_blocks;
-    s = u / p.row_blocks;
+    r = 2 * (u % p.row_pairs) + static_cast<int>(rank);
+    s = u / p.row_pairs;
     vt0 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * s / p.nsplit);
     vt1 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * (s + 1) / p.nsplit);
   };
@@ -136,33 +154,37 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      for (int u = cluster_id; u < units && ok; u += num_clusters) {
         int r, s, vt0, vt1;
         run_of(u, r, s, vt0, vt1);
         for (int vt = vt0; vt < vt1 && ok; ++vt) {
           for (int ks = 0; ks < p.ksteps; ++ks, ++it) {
             const uint32_t st = it % STAGES, ph = (it / STAGES) & 1;
             if (!(ok = mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag))) break;
-            const uint32_t fb = full0 + 8 * st;
-            mbar_arrive_expect_tx(fb, A_BYTES + B_BYTES);
-            tma_load_2d(smem_u32(smem + OFF_A + st * A_BYTES), &tmap_h, fb, ks * BK, r * BM);
-            tma_load_2d(smem_u32(smem + OFF_B + st * B_BYTES), &tmap_w, fb, ks * BK, vt * BN);
+            // the leader's barrier counts the bytes of both CTAs' loads of this stage
+            if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, 2 * (A_BYTES + B_BYTES));
+            const uint32_t fb = full_leader + 8 * st;
+            tma_load_2d_pair(smem_u32(smem + OFF_A + st * A_BYTES), &tmap_h, fb, ks * BK, r * BM);
+            tma_load_2d_pair(smem_u32(smem + OFF_B + st * B_BYTES), &tmap_w, fb, ks * BK,
+                             vt * BN + static_cast<int>(rank) * BNH);
           }
         }
       }
+      // Drain: a stage is released only after its loads landed and the MMAs that read it
+      // finished, so waiting for the release of the last stages covers both.
       const uint32_t last = it < STAGES ? it : STAGES;
       for (uint32_t j = 0; j < last; ++j) {
         const uint32_t i2 = it - 1 - j;
-        mbar_wait(full0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1, abort_flag);
+        mbar_wait(empty0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1, abort_flag);
       }
     }
   } else if (warp == 1) {
     // ---------------------- MMA issuer ----------------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(BM, BN, false, false);
+    if (rank == 0 && lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16(2 * BM, BN, false, false);
       uint32_t it = 0, tile = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      for (int u = cluster_id; u < units && ok; u += num_clusters) {
         int r, s, vt0, vt1;
         run_of(u, r, s, vt0, vt1);
         for (int vt = vt0; vt < vt1 && ok; ++vt, ++tile) {
@@ -178,12 +200,13 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             const uint32_t sb = smem_u32(smem + OFF_B + st * B_BYTES);
 #pragma unroll
             for (int k = 0; k < BK / UK; ++k) {
-              umma_bf16(d_tmem, umma_desc_sw128(sa + k * (UK * 2), 16, 1024),
-                        umma_desc_sw128(sb + k * (UK * 2), 16, 1024), idesc, (ks > 0 || k > 0) ? 1u : 0u);
+              umma_bf16_pair(d_tmem, umma_desc_sw128(sa + k * (UK * 2), 16, 1024),
+                             umma_desc_sw128(sb + k * (UK * 2), 16, 1024), idesc,
+                             (ks > 0 || k > 0) ? 1u : 0u);
             }
-            umma_commit(empty0 + 8 * st);
+            umma_commit_pair(empty0 + 8 * st);
           }
-          if (ok) umma_commit(tfull0 + 8 * buf);
+          if (ok) umma_commit_pair(tfull0 + 8 * buf);
         }
       }
     }
@@ -192,7 +215,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     if (lane == 0) {
       uint32_t zit = 0;  // sub-tile pairs issued; both halves advance together
       bool ok = true;
-      for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+      for (int u = cluster_id; u < units && ok; u += num_clusters) {
         int r, s, vt0, vt1;
         run_of(u, r, s, vt0, vt1);
         for (int vt = vt0; vt < vt1 && ok; ++vt) {
@@ -225,7 +248,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     const uint32_t swz = static_cast<uint32_t>(row_local & 7);
     uint32_t tile = 0, zit = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+    for (int u = cluster_id; u < units && ok; u += num_clusters) {
       int r, s, vt0, vt1;
       run_of(u, r, s, vt0, vt1);
       const int row = r * BM + row_local;
@@ -340,10 +363,12 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             fence_proxy_async_smem();
             named_barrier_sync(1 + half, 128);
             if (lg == 0 && lane == 0) {
-              tma_store_2d(&tmap_g, smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES),
-                           sub_col0 - p.g_col0, r * BM);
-              tma_store_commit();
-              tma_store_wait_read<0>();
+              if (r * BM < p.T) {
+                tma_store_2d(&tmap_g, smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES),
+                             sub_col0 - p.g_col0, r * BM);
+                tma_store_commit();
+                tma_store_wait_read<0>();
+              }
               mbar_arrive(zempty0 + bi);
             }
           }
@@ -351,7 +376,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         if (!ok) break;
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty0 + 8 * buf);
+        if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);
       }
       if (kMode == kForward && ok && row < p.T) {
         float* dst = p.partials + (static_cast<size_t>(2 * s + half) * kPFields) * p.T + row;
@@ -370,12 +395,15 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   }
 
   // ---------------------- teardown ----------------------
+  // Neither CTA may leave (or free tensor memory) while its peer can still send it barrier
+  // arrivals or have MMAs reading its shared memory.
   tc_fence_before_sync();
   __syncthreads();
+  cluster_sync_all();
   tc_fence_after_sync();
   if (warp == 1) {
     __syncwarp();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
   }
   if (threadIdx.x == 0 && *abort_flag != 0 && p.status != nullptr) atomicCAS(p.status, 0, kStatusTimeout);
 }

@@ -66,8 +66,8 @@ int device_info(DeviceInfo* out) {
   return NPD_OK;
 }
 
-// How many runs to cut the vocabulary tiles into so that row_blocks * nsplit work
-// units spread evenly over the SMs.  Cost = rounds of units x tiles per unit.
+// How many runs to cut the vocabulary tiles into so that row_pairs * nsplit work
+// units spread evenly over the CTA pairs.  Cost = rounds of units x tiles per unit.
 int choose_nsplit(int row_blocks, int vtiles, int sms) {
   int best = 1;
   long long best_cost = -1;
@@ -85,7 +85,7 @@ int choose_nsplit(int row_blocks, int vtiles, int sms) {
 }
 
 struct Plan {
-  int row_blocks, vtiles, nsplit, nslots;
+  int row_blocks, row_pairs, vtiles, nsplit, nslots;
   int chunk_cols;     // vocabulary columns per gradient chunk (multiple of 256)
   int nchunks;
   bool grads;
@@ -94,8 +94,9 @@ struct Plan {
 
 int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   pl->row_blocks = (a->T + 127) / 128;
+  pl->row_pairs = (a->T + 255) / 256;
   pl->vtiles = (a->V + 255) / 256;
-  pl->nsplit = choose_nsplit(pl->row_blocks, pl->vtiles, sms);
+  pl->nsplit = choose_nsplit(pl->row_pairs, pl->vtiles, std::max(sms / 2, 1));
   pl->nslots = 2 * pl->nsplit;
   pl->grads = a->d_hidden != nullptr || a->d_weight != nullptr;
   const int vpad = pl->vtiles * 256;
@@ -172,10 +173,10 @@ int launch_gemm(bool a_mn, bool b_mn, const void* A, long long lda, const void* 
   using namespace gemm_cfg;
   CUtensorMap ma, mb;
   const bool oka = a_mn ? make_map(&ma, A, gp.M, gp.K, lda, 64, 64) : make_map(&ma, A, gp.K, gp.M, lda, 64, BM);
-  const bool okb = b_mn ? make_map(&mb, B, gp.N, gp.K, ldb, 64, 64) : make_map(&mb, B, gp.K, gp.N, ldb, 64, BN);
+  const bool okb = b_mn ? make_map(&mb, B, gp.N, gp.K, ldb, 64, 64) : make_map(&mb, B, gp.K, gp.N, ldb, 64, BNH);
   if (!oka || !okb) return NPD_ECUDA;
-  const int units = ((gp.M + BM - 1) / BM) * ((gp.N + BN - 1) / BN) * gp.k_splits;
-  const int grid = std::min(units, sms);
+  const int units = ((gp.M + PM - 1) / PM) * ((gp.N + BN - 1) / BN) * gp.k_splits;
+  const int grid = 2 * std::min(units, std::max(sms / 2, 1));  // CTA pairs
   void (*k)(const CUtensorMap, const CUtensorMap, const GemmParams) = nullptr;
   if (!a_mn && !b_mn) k = gemm_bf16_kernel<false, false>;
   if (!a_mn && b_mn) k = gemm_bf16_kernel<false, true>;
@@ -193,8 +194,9 @@ int launch_kd_tile(bool tau_one, const CUtensorMap& mh, const CUtensorMap& mw, c
   using namespace kd_cfg;
   auto k = tau_one ? kd_tile_kernel<kMode, true> : kd_tile_kernel<kMode, false>;
   if (set_smem(k, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
-  const int units = kp.row_blocks * kp.nsplit;
-  k<<<std::min(units, sms), THREADS, SMEM_BYTES, st>>>(mh, mw, mt, mg, kp);
+  const int units = kp.row_pairs * kp.nsplit;
+  const int grid = 2 * std::min(units, std::max(sms / 2, 1));  // CTA pairs
+  k<<<grid, THREADS, SMEM_BYTES, st>>>(mh, mw, mt, mg, kp);
   ++g_launches;
   return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
 }
@@ -260,7 +262,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
 
   CUtensorMap mh, mw, mt;
   if (!make_map(&mh, a->hidden, a->d, a->T, a->ldh, 64, 128) ||
-      !make_map(&mw, a->weight, a->d, a->V, a->ldw, 64, 256) ||
+      !make_map(&mw, a->weight, a->d, a->V, a->ldw, 64, 128) ||
       !make_map(&mt, a->teacher, a->V, a->T, a->ldt, 64, 128))
     return NPD_ECUDA;
 
@@ -279,6 +281,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   kp.V = a->V;
   kp.ksteps = a->d / 64;
   kp.row_blocks = pl.row_blocks;
+  kp.row_pairs = pl.row_pairs;
   kp.vt_begin = 0;
   kp.vt_count = pl.vtiles;
   kp.nsplit = pl.nsplit;
