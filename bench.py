@@ -302,7 +302,9 @@ def run_ours(args):
     # dominant kernel = the launch group with the largest share of the step
     dom = max(per_kind, key=per_kind.get)
     dom_ms = per_kind[dom]
-    dom_flops = tdv2                       # each of the four tensor kernels executes 2*T*d*V FLOPs per step
+    # FLOPs per step of each tensor launch group: the forward and gradient tiles each form the
+    # logits once (2*T*d*V); the backward launch holds both contractions (dW and dH)
+    dom_flops = 2 * tdv2 if dom == "backward_gemms" else tdv2
     achieved = dom_flops / (dom_ms * 1e-3) / 1e12
     peak_tf = peaks["bf16_sustained"]      # timed inside a long step
     step_flops_alg = 3 * tdv2              # 6*T*d*V: the contractions the method defines

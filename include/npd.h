@@ -107,8 +107,8 @@ typedef struct npd_kd_args {
   /* Optional timing hooks.  HOST array of n_phase_events cudaEvent_t (as void*), or NULL.
      Event 0 is recorded on the stream before the first kernel, event i after the i-th
      launch group, in this order: forward tiles, per-token merge, then for every
-     vocabulary chunk: gradient tiles, dW contraction, dH contraction; last the dH
-     conversion if there is one.  Groups beyond n_phase_events - 1 are not recorded.
+     vocabulary chunk: gradient tiles, the dW and dH contractions (one launch); last the
+     dH conversion if there is one.  Groups beyond n_phase_events - 1 are not recorded.
      npd_phase_count() tells how many groups a call has. */
   void* const* phase_events;
   int32_t n_phase_events;

@@ -258,7 +258,7 @@ class KDStep:
         groups, chunks = npd_phase_count(self.args)
         names = ["forward_tiles", "merge"]
         for _ in range(chunks):
-            names += ["gradient_tiles", "dweight_gemm", "dhidden_gemm"]
+            names += ["gradient_tiles", "backward_gemms"]
         names += ["dhidden_convert"] * (groups - len(names))
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(groups + 1)]
         # an event only owns a CUDA handle once it has been recorded

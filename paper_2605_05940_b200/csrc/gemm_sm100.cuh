@@ -8,13 +8,18 @@
 // (memory [K][rows contiguous]); the second form lets the logit-gradient block
 // and the hidden states be read as they lie in memory, with no transposes.
 //
+// One launch runs one or two such problems.  With two, the CTA pairs first take the
+// (long) units of problem 0 and then the (short, split-K) units of problem 1, dealt
+// so that every pair ends at about the same time; this is how the dW and dH products
+// of one vocabulary chunk share a launch without a tail in between.
+//
 // Two CTAs on neighbouring SMs (a cluster of 2) work as a pair on a 256 x 256 output tile
 // with tcgen05 .cta_group::2: each CTA stages its own 128 rows of A and its own 128 of the
 // tile's 256 rows of B (32 KB per k-step per SM) and receives its own 128 output rows in
 // tensor memory.  One CTA per SM, 192 threads: warp 0 = TMA producer, warp 1 = TMEM owner
 // and, in the leader CTA (cluster rank 0), the MMA issuer of the pair, warps 2-5 = epilogue
 // (one accumulator row per thread).  6-stage operand ring, double-buffered accumulator
-// (2 x 256 TMEM columns), so the epilogue of one tile overlaps the MMAs of the next.
+// (2 x 256 TMEM columns), so the epilogue of one unit overlaps the MMAs of the next.
 #pragma once
 
 #include "ptx_sm100.cuh"
@@ -29,13 +34,21 @@ enum GemmOutMode : int {
   kOutAddBF16 = 4     // D = bf16(D + acc)
 };
 
-struct GemmParams {
+struct GemmProblem {
   int M, N, K;
-  int k_splits;   // > 1 only with kOutAtomicF32
-  void* out;
-  long long ldo;  // elements
+  int a_mn, b_mn;  // 1 = operand is MN-major
+  int k_splits;    // > 1 only with kOutAtomicF32
   int out_mode;
-  int* status;    // device status word
+  void* out;
+  long long ldo;   // elements
+};
+
+struct GemmParams {
+  GemmProblem pr[2];
+  int units[2];    // work units of each problem (tiles x k_splits); units[1] = 0 for a single problem
+  int q0, rem0;    // units[0] = q0 * pairs + rem0
+  int extra1;      // units of problem 1 that each pair WITHOUT a remainder unit of problem 0 takes first
+  int* status;     // device status word
 };
 
 namespace gemm_cfg {
@@ -49,9 +62,52 @@ constexpr int TMEM_COLS = 512;
 constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024;  // + barriers + alignment
 }  // namespace gemm_cfg
 
-template <bool kAMn, bool kBMn>
+// The i-th unit of CTA pair c out of C.  Problem-0 units go round robin.  The pairs that got
+// one unit fewer of problem 0 (c >= rem0) make up for it with `extra1` units of problem 1;
+// the rest of problem 1 goes round robin over all pairs.
+__host__ __device__ inline bool gemm_unit_at(const GemmParams& p, int c, int C, int i, int& prob, int& v) {
+  const int n0 = p.q0 + (c < p.rem0 ? 1 : 0);
+  if (i < n0) {
+    prob = 0;
+    v = c + i * C;
+    return true;
+  }
+  prob = 1;
+  int j = i - n0;
+  int base = 0;
+  if (p.rem0 > 0) {
+    const int nb = C - p.rem0;
+    base = p.extra1 * nb;
+    if (c >= p.rem0) {
+      if (j < p.extra1) {
+        v = j * nb + (c - p.rem0);
+        return v < p.units[1];
+      }
+      j -= p.extra1;
+    }
+  }
+  v = base + j * C + c;
+  return v < p.units[1];
+}
+
+struct GemmUnit {
+  int m0, n0, kt0, kt1;  // pair-tile origin and k-tile range
+};
+__device__ __forceinline__ GemmUnit gemm_decode(const GemmProblem& g, int v) {
+  using namespace gemm_cfg;
+  const int tiles_m = (g.M + PM - 1) / PM, tiles_n = (g.N + BN - 1) / BN, ktiles = (g.K + BK - 1) / BK;
+  const int ks = v / (tiles_n * tiles_m);
+  GemmUnit u;
+  u.n0 = (v % tiles_n) * BN;
+  u.m0 = ((v / tiles_n) % tiles_m) * PM;
+  u.kt0 = static_cast<int>(static_cast<long long>(ktiles) * ks / g.k_splits);
+  u.kt1 = static_cast<int>(static_cast<long long>(ktiles) * (ks + 1) / g.k_splits);
+  return u;
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(gemm_cfg::THREADS, 1)
-gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__ CUtensorMap tmap_b0,
+                 const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_b1,
                  const GemmParams p) {
   using namespace gemm_cfg;
   extern __shared__ uint8_t smem_raw[];
@@ -83,8 +139,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     }
     *abort_flag = 0;
     fence_mbar_init();
-    prefetch_tmap(&tmap_a);
-    prefetch_tmap(&tmap_b);
+    prefetch_tmap(&tmap_a0);
+    prefetch_tmap(&tmap_b0);
+    if (p.units[1] > 0) {
+      prefetch_tmap(&tmap_a1);
+      prefetch_tmap(&tmap_b1);
+    }
   }
   if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
   tc_fence_before_sync();
@@ -95,23 +155,20 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
   const uint32_t full_leader = mapa_shared(full0, 0);
   const uint32_t tempty_leader = mapa_shared(tempty0, 0);
 
-  const int tiles_m = (p.M + PM - 1) / PM;
-  const int tiles_n = (p.N + BN - 1) / BN;
-  const int ktiles = (p.K + BK - 1) / BK;
-  const int units = tiles_m * tiles_n * p.k_splits;
-
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int u = cluster_id; u < units && ok; u += num_clusters) {
-        const int n0 = (u % tiles_n) * BN + static_cast<int>(rank) * BNH;        // this CTA's B rows
-        const int m0 = ((u / tiles_n) % tiles_m) * PM + static_cast<int>(rank) * BM;  // and A rows
-        const int ks = u / (tiles_n * tiles_m);
-        const int kt0 = static_cast<int>(static_cast<long long>(ktiles) * ks / p.k_splits);
-        const int kt1 = static_cast<int>(static_cast<long long>(ktiles) * (ks + 1) / p.k_splits);
-        for (int kt = kt0; kt < kt1; ++kt, ++it) {
+      int prob, v;
+      for (int i = 0; ok && gemm_unit_at(p, cluster_id, num_clusters, i, prob, v); ++i) {
+        const GemmProblem& g = p.pr[prob];
+        const GemmUnit u = gemm_decode(g, v);
+        const CUtensorMap* ta = prob ? &tmap_a1 : &tmap_a0;
+        const CUtensorMap* tb = prob ? &tmap_b1 : &tmap_b0;
+        const int m0 = u.m0 + static_cast<int>(rank) * BM;   // this CTA's A rows
+        const int n0 = u.n0 + static_cast<int>(rank) * BNH;  // and B rows
+        for (int kt = u.kt0; kt < u.kt1; ++kt, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
           if (!(ok = mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag))) break;
           // the leader's barrier counts the bytes of both CTAs' loads of this stage
@@ -119,17 +176,17 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
           const uint32_t fb = full_leader + 8 * s;
           const uint32_t sa = smem_u32(smem_a + s * A_BYTES), sb = smem_u32(smem_b + s * B_BYTES);
           const int k0 = kt * BK;
-          if (kAMn) {
+          if (g.a_mn) {
 #pragma unroll
-            for (int i = 0; i < BM / 64; ++i) tma_load_2d_pair(sa + i * 8192, &tmap_a, fb, m0 + 64 * i, k0);
+            for (int j = 0; j < BM / 64; ++j) tma_load_2d_pair(sa + j * 8192, ta, fb, m0 + 64 * j, k0);
           } else {
-            tma_load_2d_pair(sa, &tmap_a, fb, k0, m0);
+            tma_load_2d_pair(sa, ta, fb, k0, m0);
           }
-          if (kBMn) {
+          if (g.b_mn) {
 #pragma unroll
-            for (int i = 0; i < BNH / 64; ++i) tma_load_2d_pair(sb + i * 8192, &tmap_b, fb, n0 + 64 * i, k0);
+            for (int j = 0; j < BNH / 64; ++j) tma_load_2d_pair(sb + j * 8192, tb, fb, n0 + 64 * j, k0);
           } else {
-            tma_load_2d_pair(sb, &tmap_b, fb, k0, n0);
+            tma_load_2d_pair(sb, tb, fb, k0, n0);
           }
         }
       }
@@ -144,29 +201,30 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------
     if (rank == 0 && lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16(PM, BN, kAMn, kBMn);
       uint32_t it = 0, tile = 0;
       bool ok = true;
-      for (int u = cluster_id; u < units && ok; u += num_clusters, ++tile) {
-        const int ks = u / (tiles_n * tiles_m);
-        const int kt0 = static_cast<int>(static_cast<long long>(ktiles) * ks / p.k_splits);
-        const int kt1 = static_cast<int>(static_cast<long long>(ktiles) * (ks + 1) / p.k_splits);
+      int prob, v;
+      for (int i = 0; ok && gemm_unit_at(p, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
+        const GemmProblem& g = p.pr[prob];
+        const GemmUnit u = gemm_decode(g, v);
+        const uint32_t idesc = umma_idesc_bf16(PM, BN, g.a_mn != 0, g.b_mn != 0);
         const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
         if (!(ok = mbar_wait(tempty0 + 8 * buf, tph ^ 1, abort_flag))) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + buf * BN;
-        for (int kt = kt0; kt < kt1; ++kt, ++it) {
+        // byte step between the four K=16 slices of a stage, and the descriptor's leading offset
+        const uint32_t a_step = g.a_mn ? UK * 128 : UK * 2, a_lbo = g.a_mn ? BK * 128 : 16;
+        const uint32_t b_step = g.b_mn ? UK * 128 : UK * 2, b_lbo = g.b_mn ? BK * 128 : 16;
+        for (int kt = u.kt0; kt < u.kt1; ++kt, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
           if (!(ok = mbar_wait(full0 + 8 * s, ph, abort_flag))) break;
           tc_fence_after_sync();
           const uint32_t sa = smem_u32(smem_a + s * A_BYTES), sb = smem_u32(smem_b + s * B_BYTES);
 #pragma unroll
           for (int k = 0; k < BK / UK; ++k) {
-            const uint64_t da = kAMn ? umma_desc_sw128(sa + k * (UK * 128), BK * 128, 1024)
-                                     : umma_desc_sw128(sa + k * (UK * 2), 16, 1024);
-            const uint64_t db = kBMn ? umma_desc_sw128(sb + k * (UK * 128), BK * 128, 1024)
-                                     : umma_desc_sw128(sb + k * (UK * 2), 16, 1024);
-            umma_bf16_pair(d_tmem, da, db, idesc, (kt > kt0 || k > 0) ? 1u : 0u);
+            umma_bf16_pair(d_tmem, umma_desc_sw128(sa + k * a_step, a_lbo, 1024),
+                           umma_desc_sw128(sb + k * b_step, b_lbo, 1024), idesc,
+                           (kt > u.kt0 || k > 0) ? 1u : 0u);
           }
           umma_commit_pair(empty0 + 8 * s);
         }
@@ -178,9 +236,13 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
     const int lg = warp & 3;  // TMEM lane group this warp may read
     uint32_t tile = 0;
     bool ok = true;
-    for (int u = cluster_id; u < units && ok; u += num_clusters, ++tile) {
-      const int n0 = (u % tiles_n) * BN;
-      const int m0 = ((u / tiles_n) % tiles_m) * PM + static_cast<int>(rank) * BM;
+    int prob, v;
+    for (int i = 0; ok && gemm_unit_at(p, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
+      const GemmProblem& g = p.pr[prob];
+      const GemmUnit u = gemm_decode(g, v);
+      const int n0 = u.n0;
+      const int m0 = u.m0 + static_cast<int>(rank) * BM;
+      const int out_mode = g.out_mode;
       const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
       if (!(ok = mbar_wait(tfull0 + 8 * buf, tph, abort_flag))) break;
       tc_fence_after_sync();
@@ -188,45 +250,46 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN;
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
+        const int col0 = n0 + c * 32;
+        if (col0 >= g.N) break;  // uniform over the warp
         uint32_t r[32];
         tmem_ld32(taddr + c * 32, r);
         tmem_ld_wait();
-        const int col0 = n0 + c * 32;
-        if (row < p.M && col0 < p.N) {
-          const bool full_chunk = (col0 + 32 <= p.N);
-          if (p.out_mode == kOutStoreBF16 || p.out_mode == kOutAddBF16) {
-            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(p.out) + row * p.ldo + col0;
+        if (row < g.M) {
+          const bool full_chunk = (col0 + 32 <= g.N);
+          if (out_mode == kOutStoreBF16 || out_mode == kOutAddBF16) {
+            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(g.out) + row * g.ldo + col0;
             if (full_chunk) {
               uint4* o4 = reinterpret_cast<uint4*>(o);
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                float v[8];
+                float x[8];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) v[q] = __uint_as_float(r[8 * j + q]);
-                if (p.out_mode == kOutAddBF16) {
+                for (int q = 0; q < 8; ++q) x[q] = __uint_as_float(r[8 * j + q]);
+                if (out_mode == kOutAddBF16) {
                   const uint4 old = o4[j];
-                  v[0] += bf16_lo(old.x); v[1] += bf16_hi(old.x);
-                  v[2] += bf16_lo(old.y); v[3] += bf16_hi(old.y);
-                  v[4] += bf16_lo(old.z); v[5] += bf16_hi(old.z);
-                  v[6] += bf16_lo(old.w); v[7] += bf16_hi(old.w);
+                  x[0] += bf16_lo(old.x); x[1] += bf16_hi(old.x);
+                  x[2] += bf16_lo(old.y); x[3] += bf16_hi(old.y);
+                  x[4] += bf16_lo(old.z); x[5] += bf16_hi(old.z);
+                  x[6] += bf16_lo(old.w); x[7] += bf16_hi(old.w);
                 }
                 uint4 w;
-                w.x = pack_bf16x2(v[0], v[1]);
-                w.y = pack_bf16x2(v[2], v[3]);
-                w.z = pack_bf16x2(v[4], v[5]);
-                w.w = pack_bf16x2(v[6], v[7]);
+                w.x = pack_bf16x2(x[0], x[1]);
+                w.y = pack_bf16x2(x[2], x[3]);
+                w.z = pack_bf16x2(x[4], x[5]);
+                w.w = pack_bf16x2(x[6], x[7]);
                 o4[j] = w;
               }
             } else {
-              for (int j = 0; j < 32 && col0 + j < p.N; ++j) {
-                float v = __uint_as_float(r[j]);
-                if (p.out_mode == kOutAddBF16) v += __bfloat162float(o[j]);
-                o[j] = __float2bfloat16_rn(v);
+              for (int j = 0; j < 32 && col0 + j < g.N; ++j) {
+                float x = __uint_as_float(r[j]);
+                if (out_mode == kOutAddBF16) x += __bfloat162float(o[j]);
+                o[j] = __float2bfloat16_rn(x);
               }
             }
           } else {
-            float* o = reinterpret_cast<float*>(p.out) + row * p.ldo + col0;
-            if (p.out_mode == kOutAtomicF32) {
+            float* o = reinterpret_cast<float*>(g.out) + row * g.ldo + col0;
+            if (out_mode == kOutAtomicF32) {
               if (full_chunk) {
 #pragma unroll
                 for (int j = 0; j < 32; j += 4)
@@ -235,25 +298,25 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_consta
                                "f"(__uint_as_float(r[j + 2])), "f"(__uint_as_float(r[j + 3]))
                                : "memory");
               } else {
-                for (int j = 0; j < 32 && col0 + j < p.N; ++j) atomicAdd(o + j, __uint_as_float(r[j]));
+                for (int j = 0; j < 32 && col0 + j < g.N; ++j) atomicAdd(o + j, __uint_as_float(r[j]));
               }
             } else if (full_chunk) {
               float4* o4 = reinterpret_cast<float4*>(o);
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
-                float4 v = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
+                float4 x = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
                                        __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-                if (p.out_mode == kOutAddF32) {
+                if (out_mode == kOutAddF32) {
                   const float4 old = o4[j];
-                  v.x += old.x; v.y += old.y; v.z += old.z; v.w += old.w;
+                  x.x += old.x; x.y += old.y; x.z += old.z; x.w += old.w;
                 }
-                o4[j] = v;
+                o4[j] = x;
               }
             } else {
-              for (int j = 0; j < 32 && col0 + j < p.N; ++j) {
-                float v = __uint_as_float(r[j]);
-                if (p.out_mode == kOutAddF32) v += o[j];
-                o[j] = v;
+              for (int j = 0; j < 32 && col0 + j < g.N; ++j) {
+                float x = __uint_as_float(r[j]);
+                if (out_mode == kOutAddF32) x += o[j];
+                o[j] = x;
               }
             }
           }

@@ -88,6 +88,8 @@ struct Plan {
   int row_blocks, row_pairs, vtiles, nsplit, nslots;
   int chunk_cols;     // vocabulary columns per gradient chunk (multiple of 256)
   int nchunks;
+  int dh_ksplits;     // split-K of the dH product of a full chunk
+  bool dh_direct;     // dH stored straight to the output (one chunk, no split-K); else fp32 atomics
   bool grads;
   size_t off_status, off_partials, off_lse_a, off_lse_b, off_coef, off_g, off_dh, total;
 };
@@ -99,11 +101,24 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   pl->nsplit = choose_nsplit(pl->row_pairs, pl->vtiles, std::max(sms / 2, 1));
   pl->nslots = 2 * pl->nsplit;
   pl->grads = a->d_hidden != nullptr || a->d_weight != nullptr;
-  const int vpad = pl->vtiles * 256;
-  int cc = a->grad_chunk_cols > 0 ? a->grad_chunk_cols : 4096;
-  cc = std::min((cc + 255) / 256 * 256, vpad);
-  pl->chunk_cols = cc;
-  pl->nchunks = (vpad + cc - 1) / cc;
+  // Vocabulary chunks of the backward: the bf16 logit-gradient block [T, chunk_cols] is the only
+  // thing that travels between the gradient tiles and the two contractions.  Default: the
+  // largest chunk whose block stays within 256 MiB, chunks of (almost) equal width.
+  const long long budget = 256ll << 20;
+  int max_tiles = a->grad_chunk_cols > 0
+                      ? (a->grad_chunk_cols + 255) / 256
+                      : static_cast<int>(std::max<long long>(8, budget / (512ll * a->T)));
+  max_tiles = std::max(1, std::min(max_tiles, pl->vtiles));
+  pl->nchunks = (pl->vtiles + max_tiles - 1) / max_tiles;
+  const int chunk_tiles = (pl->vtiles + pl->nchunks - 1) / pl->nchunks;
+  pl->chunk_cols = chunk_tiles * 256;
+  pl->nchunks = (pl->vtiles + chunk_tiles - 1) / chunk_tiles;
+  const int cc = pl->chunk_cols;
+  // dH = G W is cut along the chunk's columns into units of about 48 k-steps so that the
+  // pairs can be filled evenly; the partial products are added with fp32 atomics.
+  const int ksteps_h = cc / 64;
+  pl->dh_ksplits = std::max(1, std::min(16, (ksteps_h + 24) / 48));
+  pl->dh_direct = pl->nchunks == 1 && pl->dh_ksplits == 1;
   size_t off = 0;
   pl->off_status = off;
   off += 1024;
@@ -120,7 +135,7 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   if (pl->grads) {
     off = align_up(off + 2 * static_cast<size_t>(a->T) * cc, 1024);
     pl->off_dh = off;
-    if (pl->nchunks > 1) off = align_up(off + sizeof(float) * static_cast<size_t>(a->T) * a->d, 1024);
+    if (!pl->dh_direct) off = align_up(off + sizeof(float) * static_cast<size_t>(a->T) * a->d, 1024);
   }
   pl->total = off;
   return NPD_OK;
@@ -168,22 +183,50 @@ int set_smem(K kernel, int bytes) {
              : NPD_ECUDA;
 }
 
-int launch_gemm(bool a_mn, bool b_mn, const void* A, long long lda, const void* B, long long ldb,
-                const GemmParams& gp, int sms, cudaStream_t st) {
+struct GemmOperands {
+  const void* A;
+  long long lda;
+  const void* B;
+  long long ldb;
+};
+
+// k-steps one unit of a problem runs (its cost in the schedule)
+int gemm_unit_ksteps(const GemmProblem& g) {
+  return std::max(1, ((g.K + gemm_cfg::BK - 1) / gemm_cfg::BK + g.k_splits - 1) / g.k_splits);
+}
+int gemm_units(const GemmProblem& g) {
   using namespace gemm_cfg;
-  CUtensorMap ma, mb;
-  const bool oka = a_mn ? make_map(&ma, A, gp.M, gp.K, lda, 64, 64) : make_map(&ma, A, gp.K, gp.M, lda, 64, BM);
-  const bool okb = b_mn ? make_map(&mb, B, gp.N, gp.K, ldb, 64, 64) : make_map(&mb, B, gp.K, gp.N, ldb, 64, BNH);
-  if (!oka || !okb) return NPD_ECUDA;
-  const int units = ((gp.M + PM - 1) / PM) * ((gp.N + BN - 1) / BN) * gp.k_splits;
-  const int grid = 2 * std::min(units, std::max(sms / 2, 1));  // CTA pairs
-  void (*k)(const CUtensorMap, const CUtensorMap, const GemmParams) = nullptr;
-  if (!a_mn && !b_mn) k = gemm_bf16_kernel<false, false>;
-  if (!a_mn && b_mn) k = gemm_bf16_kernel<false, true>;
-  if (a_mn && !b_mn) k = gemm_bf16_kernel<true, false>;
-  if (a_mn && b_mn) k = gemm_bf16_kernel<true, true>;
-  if (set_smem(k, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
-  k<<<grid, THREADS, SMEM_BYTES, st>>>(ma, mb, gp);
+  return ((g.M + PM - 1) / PM) * ((g.N + BN - 1) / BN) * g.k_splits;
+}
+
+// One launch for one or two problems (see gemm_sm100.cuh for how the units are dealt).
+int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, int* status, int sms,
+                cudaStream_t st) {
+  using namespace gemm_cfg;
+  CUtensorMap maps[4];
+  GemmParams gp{};
+  for (int i = 0; i < 2; ++i) {
+    const int j = i < nprob ? i : 0;  // an unused slot repeats problem 0's (valid) maps
+    const GemmProblem& g = pr[j];
+    const bool oka = g.a_mn ? make_map(&maps[2 * i], ops[j].A, g.M, g.K, ops[j].lda, 64, 64)
+                            : make_map(&maps[2 * i], ops[j].A, g.K, g.M, ops[j].lda, 64, BM);
+    const bool okb = g.b_mn ? make_map(&maps[2 * i + 1], ops[j].B, g.N, g.K, ops[j].ldb, 64, 64)
+                            : make_map(&maps[2 * i + 1], ops[j].B, g.K, g.N, ops[j].ldb, 64, BNH);
+    if (!oka || !okb) return NPD_ECUDA;
+    gp.pr[i] = g;
+    gp.units[i] = i < nprob ? gemm_units(g) : 0;
+  }
+  const int pairs = std::max(1, std::min(gp.units[0] + gp.units[1], std::max(sms / 2, 1)));
+  gp.q0 = gp.units[0] / pairs;
+  gp.rem0 = gp.units[0] % pairs;
+  gp.extra1 = 0;
+  if (nprob == 2 && gp.rem0 > 0) {
+    const int c0 = gemm_unit_ksteps(pr[0]), c1 = gemm_unit_ksteps(pr[1]);
+    gp.extra1 = std::min((c0 + c1 / 2) / c1, gp.units[1] / (pairs - gp.rem0));
+  }
+  gp.status = status;
+  if (set_smem(gemm_bf16_kernel, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
+  gemm_bf16_kernel<<<2 * pairs, THREADS, SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], gp);
   ++g_launches;
   return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
 }
@@ -328,6 +371,9 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   __nv_bfloat16* gbuf = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_g);
   float* dh_acc = reinterpret_cast<float*>(ws + pl.off_dh);
   const long long ldg = pl.chunk_cols;
+  if (!pl.dh_direct &&
+      cudaMemsetAsync(dh_acc, 0, sizeof(float) * static_cast<size_t>(a->T) * a->d, st) != cudaSuccess)
+    return NPD_ECUDA;
   for (int c = 0; c < pl.nchunks; ++c) {
     const int col0 = c * pl.chunk_cols;
     const int cols = std::min(pl.chunk_cols, a->V - col0);  // columns of this chunk inside V
@@ -347,45 +393,47 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     if ((rc = launch_kd_tile<kGradient>(tau_one, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
     rec.mark();
 
+    GemmProblem pr[2] = {};
+    GemmOperands ops[2] = {};
     // dW[col0 .. col0+cols) = G_chunk^T H       (M = vocabulary rows, N = d, K = T)
-    GemmParams gw{};
-    gw.M = cols;
-    gw.N = a->d;
-    gw.K = a->T;
-    gw.k_splits = 1;
-    gw.ldo = a->ldw;
-    gw.status = status;
+    pr[0].M = cols;
+    pr[0].N = a->d;
+    pr[0].K = a->T;
+    pr[0].a_mn = 1;
+    pr[0].b_mn = 1;
+    pr[0].k_splits = 1;
+    pr[0].ldo = a->ldw;
     if (a->d_weight_dtype == NPD_DTYPE_F32) {
-      gw.out = static_cast<float*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw;
-      gw.out_mode = (a->flags & NPD_KD_ACCUMULATE_DW) ? kOutAddF32 : kOutStoreF32;
+      pr[0].out = static_cast<float*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw;
+      pr[0].out_mode = (a->flags & NPD_KD_ACCUMULATE_DW) ? kOutAddF32 : kOutStoreF32;
     } else {
-      gw.out = static_cast<__nv_bfloat16*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw;
-      gw.out_mode = kOutStoreBF16;
+      pr[0].out = static_cast<__nv_bfloat16*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw;
+      pr[0].out_mode = kOutStoreBF16;
     }
-    if ((rc = launch_gemm(true, true, gbuf, ldg, a->hidden, a->ldh, gw, di.sms, st)) != NPD_OK) return rc;
-    rec.mark();
-
+    ops[0] = {gbuf, ldg, a->hidden, a->ldh};
     // dH (+)= G_chunk W[col0 .. col0+cols)      (M = T, N = d, K = vocabulary rows of the chunk)
-    GemmParams gh{};
-    gh.M = a->T;
-    gh.N = a->d;
-    gh.K = cols;
-    gh.k_splits = 1;
-    gh.status = status;
-    if (pl.nchunks == 1) {
-      gh.out = a->d_hidden;
-      gh.ldo = a->ldh;
-      gh.out_mode = kOutStoreBF16;
+    pr[1].M = a->T;
+    pr[1].N = a->d;
+    pr[1].K = cols;
+    pr[1].a_mn = 0;
+    pr[1].b_mn = 1;
+    if (pl.dh_direct) {
+      pr[1].k_splits = 1;
+      pr[1].out = a->d_hidden;
+      pr[1].ldo = a->ldh;
+      pr[1].out_mode = kOutStoreBF16;
     } else {
-      gh.out = dh_acc;
-      gh.ldo = a->d;
-      gh.out_mode = c == 0 ? kOutStoreF32 : kOutAddF32;
+      pr[1].k_splits = std::max(1, std::min(pl.dh_ksplits, (cols + 63) / 64));
+      pr[1].out = dh_acc;
+      pr[1].ldo = a->d;
+      pr[1].out_mode = kOutAtomicF32;
     }
-    const __nv_bfloat16* wc = static_cast<const __nv_bfloat16*>(a->weight) + static_cast<size_t>(col0) * a->ldw;
-    if ((rc = launch_gemm(false, true, gbuf, ldg, wc, a->ldw, gh, di.sms, st)) != NPD_OK) return rc;
+    ops[1] = {gbuf, ldg, static_cast<const __nv_bfloat16*>(a->weight) + static_cast<size_t>(col0) * a->ldw,
+              a->ldw};
+    if ((rc = launch_gemm(2, pr, ops, status, di.sms, st)) != NPD_OK) return rc;
     rec.mark();
   }
-  if (pl.nchunks > 1) {
+  if (!pl.dh_direct) {
     const long long n = static_cast<long long>(a->T) * (a->d / 8);
     f32_to_bf16_rows_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(
         dh_acc, a->T, a->d, static_cast<__nv_bfloat16*>(a->d_hidden), a->ldh);
@@ -408,7 +456,7 @@ int npd_phase_count(const npd_kd_args* args, int32_t* out_groups, int32_t* out_c
   if (pl.grads)
     for (int c = 0; c < pl.nchunks; ++c)
       if (args->V - c * pl.chunk_cols > 0) ++chunks;
-  *out_groups = 2 + 3 * chunks + ((pl.grads && pl.nchunks > 1) ? 1 : 0);
+  *out_groups = 2 + 2 * chunks + ((pl.grads && !pl.dh_direct) ? 1 : 0);
   if (out_chunks != nullptr) *out_chunks = chunks;
   return NPD_OK;
 }
@@ -559,17 +607,18 @@ int npd_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, i
   int rc = device_info(&di);
   if (rc != NPD_OK) return rc;
   if (di.cc_major != 10) return NPD_EARCH;
-  GemmParams gp{};
-  gp.M = M;
-  gp.N = N;
-  gp.K = K;
-  gp.k_splits = k_splits;
-  gp.out = out;
-  gp.ldo = ldo;
-  gp.out_mode = out_mode;
-  gp.status = nullptr;
-  return launch_gemm(a_mn_major != 0, b_mn_major != 0, A, lda, B, ldb, gp, di.sms,
-                     static_cast<cudaStream_t>(cuda_stream));
+  GemmProblem pr{};
+  pr.M = M;
+  pr.N = N;
+  pr.K = K;
+  pr.a_mn = a_mn_major != 0;
+  pr.b_mn = b_mn_major != 0;
+  pr.k_splits = k_splits;
+  pr.out = out;
+  pr.ldo = ldo;
+  pr.out_mode = out_mode;
+  const GemmOperands ops{A, lda, B, ldb};
+  return launch_gemm(1, &pr, &ops, nullptr, di.sms, static_cast<cudaStream_t>(cuda_stream));
 }
 
 }  // extern "C"
