@@ -228,11 +228,10 @@ int npd_kd_forward_noalloc(const npd_kd_args* args, void* cuda_stream, int32_t* 
 
 /* out_mode of npd_gemm_bf16 */
 enum {
-  NPD_GEMM_STORE_F32 = 0,  /* D = acc                       */
-  NPD_GEMM_ADD_F32 = 1,    /* D += acc (one owner per tile) */
-  NPD_GEMM_STORE_BF16 = 2, /* D = bf16(acc)                 */
-  NPD_GEMM_ATOMIC_F32 = 3, /* D += acc with atomics (split-K; D must be initialised) */
-  NPD_GEMM_ADD_BF16 = 4    /* D = bf16(D + acc)             */
+  NPD_GEMM_STORE_F32 = 0,  /* D = acc                                                  */
+  NPD_GEMM_ADD_F32 = 1,    /* D += acc, element-wise atomic adds (D must be initialised) */
+  NPD_GEMM_STORE_BF16 = 2, /* D = bf16(acc)                                            */
+  NPD_GEMM_ATOMIC_F32 = 3  /* same as NPD_GEMM_ADD_F32; the mode split-K is meant for   */
 };
 
 /*
@@ -242,7 +241,9 @@ enum {
  *     D[M,N] (+)= sum_k A[m,k] * B[n,k]      bf16 inputs, fp32 accumulation.
  * An operand is K-major (memory [rows][K], x_mn_major = 0, ld >= K) or MN-major
  * (memory [K][rows], x_mn_major = 1, ld >= rows).  Pointers 16-byte aligned, row
- * strides multiples of 8 elements.  k_splits > 1 needs NPD_GEMM_ATOMIC_F32.
+ * strides multiples of 16 bytes.  k_splits > 1 needs one of the two adding modes;
+ * the order of the additions, and so the last bits of the sums, can differ from
+ * run to run.
  */
 int npd_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, int32_t a_mn_major,
                   const void* B, int64_t ldb, int32_t b_mn_major, void* out, int64_t ldo,

@@ -22,7 +22,7 @@ NPD_EWORKSPACE, NPD_ECUDA, NPD_ETIMEOUT, NPD_EUNSUPPORTED = -6, -7, -8, -9
 NPD_DTYPE_BF16, NPD_DTYPE_F32 = 0, 1
 NPD_KD_ACCUMULATE_DW = 1
 NPD_SELECT_TEACHER_IFD_LE_1 = 1
-NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32, NPD_GEMM_ADD_BF16 = range(5)
+NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32 = range(4)
 
 EXPORTS = ("npd_workspace_bytes", "npd_phase_count", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
            "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16",

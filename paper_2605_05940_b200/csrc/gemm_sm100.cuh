@@ -13,34 +13,32 @@
 // so that every pair ends at about the same time; this is how the dW and dH products
 // of one vocabulary chunk share a launch without a tail in between.
 //
-// Two CTAs on neighbouring SMs (a cluster of 2) work as a pair on a 256 x 256 output tile
-// with tcgen05 .cta_group::2: each CTA stages its own 128 rows of A and its own 128 of the
-// tile's 256 rows of B (32 KB per k-step per SM) and receives its own 128 output rows in
-// tensor memory.  One CTA per SM, 192 threads: warp 0 = TMA producer, warp 1 = TMEM owner
-// and, in the leader CTA (cluster rank 0), the MMA issuer of the pair, warps 2-5 = epilogue
-// (one accumulator row per thread).  6-stage operand ring, double-buffered accumulator
-// (2 x 256 TMEM columns), so the epilogue of one unit overlaps the MMAs of the next.
+// Two CTAs on neighbouring SMs (a cluster of 2) work as a pair on a 256 x 512 output tile
+// with tcgen05 .cta_group::2 (two M=256, N=256 accumulators that share the A operand): per
+// k-step each CTA stages its own 128 rows of A and its own half (128 rows) of each of the two
+// 256-row blocks of B, 48 KB for 2 x 128 x 256 x 64 MACs per SM.  The kernels here are bound by
+// the L2-to-SM operand traffic, and this tile moves a quarter fewer bytes per MAC than a
+// 256 x 256 pair tile; the price is that the 512 accumulator columns fill tensor memory, so
+// the drain of a tile is not overlapped with the next tile's MMAs (a few per cent at the
+// k-extents used here).
+//
+// One CTA per SM, 320 threads: warp 0 = TMA producer, warp 1 = TMEM owner and, in the leader
+// CTA (cluster rank 0), the MMA issuer of the pair, warps 2-9 = epilogue in two groups of
+// four warps (one accumulator row per thread, each group drains half of the columns):
+// TMEM -> registers -> 128-byte-swizzled shared memory -> TMA store, or TMA reduce-add for
+// outputs that are accumulated (split-K, or several launches adding into one matrix).
 #pragma once
 
 #include "ptx_sm100.cuh"
 
 namespace npd {
 
-enum GemmOutMode : int {
-  kOutStoreF32 = 0,   // D = acc
-  kOutAddF32 = 1,     // D += acc (plain read-modify-write; each tile has one owner)
-  kOutStoreBF16 = 2,  // D = bf16(acc)
-  kOutAtomicF32 = 3,  // D += acc with red.global.add (split-K)
-  kOutAddBF16 = 4     // D = bf16(D + acc)
-};
-
 struct GemmProblem {
   int M, N, K;
   int a_mn, b_mn;  // 1 = operand is MN-major
-  int k_splits;    // > 1 only with kOutAtomicF32
-  int out_mode;
-  void* out;
-  long long ldo;   // elements
+  int k_splits;    // > 1 only with out_reduce
+  int out_f32;     // output elements: 1 = fp32, 0 = bf16
+  int out_reduce;  // 1 = D += acc (atomic, any number of adders), 0 = D = acc
 };
 
 struct GemmParams {
@@ -52,14 +50,23 @@ struct GemmParams {
 };
 
 namespace gemm_cfg {
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 6, UK = 16;  // BM = rows per CTA (256 per pair)
-constexpr int PM = 2 * BM;            // rows of a pair tile
-constexpr int BNH = BN / 2;           // B rows each CTA of the pair stages
-constexpr int A_BYTES = BM * BK * 2;  // 16 KB
-constexpr int B_BYTES = BNH * BK * 2; // 16 KB
-constexpr int THREADS = 192;
+constexpr int BM = 128;                 // rows per CTA
+constexpr int PM = 2 * BM;              // rows of a pair tile
+constexpr int BNS = 256;                // columns of one accumulator (the MMA's N)
+constexpr int NSUB = 2;                 // accumulators per tile
+constexpr int BN = BNS * NSUB;          // columns of a pair tile
+constexpr int BK = 64, UK = 16, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;             // 16 KB
+constexpr int BSUB_BYTES = (BNS / 2) * BK * 2;   // 16 KB: this CTA's half of one 256-row block of B
+constexpr int B_BYTES = NSUB * BSUB_BYTES;       // 32 KB
+constexpr int OUT_BYTES = 128 * 128;             // staging of one epilogue group: 128 rows x 128 B
+constexpr int THREADS = 320;
 constexpr int TMEM_COLS = 512;
-constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024;  // + barriers + alignment
+constexpr int OFF_A = 0;
+constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
+constexpr int OFF_OUT = OFF_B + STAGES * B_BYTES;
+constexpr int OFF_BAR = OFF_OUT + 2 * OUT_BYTES;
+constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;  // + barriers + alignment
 }  // namespace gemm_cfg
 
 // The i-th unit of CTA pair c out of C.  Problem-0 units go round robin.  The pairs that got
@@ -92,6 +99,7 @@ __host__ __device__ inline bool gemm_unit_at(const GemmParams& p, int c, int C, 
 
 struct GemmUnit {
   int m0, n0, kt0, kt1;  // pair-tile origin and k-tile range
+  int ns;                // accumulators in use: 2, or 1 when the tile's second 256 columns lie beyond N
 };
 __device__ __forceinline__ GemmUnit gemm_decode(const GemmProblem& g, int v) {
   using namespace gemm_cfg;
@@ -102,22 +110,24 @@ __device__ __forceinline__ GemmUnit gemm_decode(const GemmProblem& g, int v) {
   u.m0 = ((v / tiles_n) % tiles_m) * PM;
   u.kt0 = static_cast<int>(static_cast<long long>(ktiles) * ks / g.k_splits);
   u.kt1 = static_cast<int>(static_cast<long long>(ktiles) * (ks + 1) / g.k_splits);
+  u.ns = (g.N - u.n0 > BNS) ? 2 : 1;
   return u;
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(gemm_cfg::THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__ CUtensorMap tmap_b0,
-                 const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_b1,
+                 const __grid_constant__ CUtensorMap tmap_o0, const __grid_constant__ CUtensorMap tmap_a1,
+                 const __grid_constant__ CUtensorMap tmap_b1, const __grid_constant__ CUtensorMap tmap_o1,
                  const GemmParams p) {
   using namespace gemm_cfg;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
-  uint8_t* smem_a = smem;
-  uint8_t* smem_b = smem + STAGES * A_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_BYTES + B_BYTES));
-  // bars[0..S) full, [S..2S) empty, [2S..2S+2) tmem full, [2S+2..2S+4) tmem empty
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  uint8_t* smem_a = smem + OFF_A;
+  uint8_t* smem_b = smem + OFF_B;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
+  // bars[0..S) full, [S..2S) empty, [2S] tmem full, [2S+1] tmem empty
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5;
@@ -126,24 +136,24 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
   const int cluster_id = blockIdx.x >> 1;
   const int num_clusters = gridDim.x >> 1;
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
-  const uint32_t tfull0 = smem_u32(bars + 2 * STAGES), tempty0 = smem_u32(bars + 2 * STAGES + 2);
+  const uint32_t tfull = smem_u32(bars + 2 * STAGES), tempty = smem_u32(bars + 2 * STAGES + 1);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(tfull0 + 8 * b, 1);
-      mbar_init(tempty0 + 8 * b, 8);  // 4 epilogue warps of each CTA, counted in the leader
-    }
+    mbar_init(tfull, 1);
+    mbar_init(tempty, 16);  // 8 epilogue warps of each CTA, counted in the leader
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmap_a0);
     prefetch_tmap(&tmap_b0);
+    prefetch_tmap(&tmap_o0);
     if (p.units[1] > 0) {
       prefetch_tmap(&tmap_a1);
       prefetch_tmap(&tmap_b1);
+      prefetch_tmap(&tmap_o1);
     }
   }
   if (warp == 1) tmem_alloc_pair(smem_u32(tmem_slot), TMEM_COLS);
@@ -153,7 +163,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t full_leader = mapa_shared(full0, 0);
-  const uint32_t tempty_leader = mapa_shared(tempty0, 0);
+  const uint32_t tempty_leader = mapa_shared(tempty, 0);
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -166,13 +176,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
         const GemmUnit u = gemm_decode(g, v);
         const CUtensorMap* ta = prob ? &tmap_a1 : &tmap_a0;
         const CUtensorMap* tb = prob ? &tmap_b1 : &tmap_b0;
-        const int m0 = u.m0 + static_cast<int>(rank) * BM;   // this CTA's A rows
-        const int n0 = u.n0 + static_cast<int>(rank) * BNH;  // and B rows
+        const int m0 = u.m0 + static_cast<int>(rank) * BM;          // this CTA's A rows
+        const int n0 = u.n0 + static_cast<int>(rank) * (BNS / 2);   // its B rows within each 256-row block
+        const uint32_t stage_bytes = 2 * (A_BYTES + u.ns * BSUB_BYTES);
         for (int kt = u.kt0; kt < u.kt1; ++kt, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1;
           if (!(ok = mbar_wait(empty0 + 8 * s, ph ^ 1, abort_flag))) break;
           // the leader's barrier counts the bytes of both CTAs' loads of this stage
-          if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * s, 2 * (A_BYTES + B_BYTES));
+          if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * s, stage_bytes);
           const uint32_t fb = full_leader + 8 * s;
           const uint32_t sa = smem_u32(smem_a + s * A_BYTES), sb = smem_u32(smem_b + s * B_BYTES);
           const int k0 = kt * BK;
@@ -182,11 +193,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
           } else {
             tma_load_2d_pair(sa, ta, fb, k0, m0);
           }
-          if (g.b_mn) {
+          for (int h = 0; h < u.ns; ++h) {
+            const uint32_t sbh = sb + h * BSUB_BYTES;
+            const int nh = n0 + h * BNS;
+            if (g.b_mn) {
 #pragma unroll
-            for (int j = 0; j < BNH / 64; ++j) tma_load_2d_pair(sb + j * 8192, tb, fb, n0 + 64 * j, k0);
-          } else {
-            tma_load_2d_pair(sb, tb, fb, k0, n0);
+              for (int j = 0; j < BNS / 2 / 64; ++j) tma_load_2d_pair(sbh + j * 8192, tb, fb, nh + 64 * j, k0);
+            } else {
+              tma_load_2d_pair(sbh, tb, fb, k0, nh);
+            }
           }
         }
       }
@@ -207,11 +222,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
       for (int i = 0; ok && gemm_unit_at(p, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
         const GemmProblem& g = p.pr[prob];
         const GemmUnit u = gemm_decode(g, v);
-        const uint32_t idesc = umma_idesc_bf16(PM, BN, g.a_mn != 0, g.b_mn != 0);
-        const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
-        if (!(ok = mbar_wait(tempty0 + 8 * buf, tph ^ 1, abort_flag))) break;
+        const uint32_t idesc = umma_idesc_bf16(PM, BNS, g.a_mn != 0, g.b_mn != 0);
+        // the accumulators are free once every epilogue warp of the pair has read the last tile
+        if (!(ok = mbar_wait(tempty, (tile & 1) ^ 1, abort_flag))) break;
         tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + buf * BN;
         // byte step between the four K=16 slices of a stage, and the descriptor's leading offset
         const uint32_t a_step = g.a_mn ? UK * 128 : UK * 2, a_lbo = g.a_mn ? BK * 128 : 16;
         const uint32_t b_step = g.b_mn ? UK * 128 : UK * 2, b_lbo = g.b_mn ? BK * 128 : 16;
@@ -222,110 +236,94 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
           const uint32_t sa = smem_u32(smem_a + s * A_BYTES), sb = smem_u32(smem_b + s * B_BYTES);
 #pragma unroll
           for (int k = 0; k < BK / UK; ++k) {
-            umma_bf16_pair(d_tmem, umma_desc_sw128(sa + k * a_step, a_lbo, 1024),
-                           umma_desc_sw128(sb + k * b_step, b_lbo, 1024), idesc,
-                           (kt > u.kt0 || k > 0) ? 1u : 0u);
+            const uint64_t da = umma_desc_sw128(sa + k * a_step, a_lbo, 1024);
+            const uint32_t acc = (kt > u.kt0 || k > 0) ? 1u : 0u;
+            umma_bf16_pair(tmem_base, da, umma_desc_sw128(sb + k * b_step, b_lbo, 1024), idesc, acc);
+            if (u.ns == 2)
+              umma_bf16_pair(tmem_base + BNS, da, umma_desc_sw128(sb + BSUB_BYTES + k * b_step, b_lbo, 1024),
+                             idesc, acc);
           }
           umma_commit_pair(empty0 + 8 * s);
         }
-        if (ok) umma_commit_pair(tfull0 + 8 * buf);
+        if (ok) umma_commit_pair(tfull);
       }
     }
   } else {
     // ------------------------------ epilogue ----------------------------------
-    const int lg = warp & 3;  // TMEM lane group this warp may read
+    const int e = warp - 2;
+    const int lg = warp & 3;   // TMEM lane group this warp may read
+    const int grp = e >> 2;    // epilogue group: which half of the tile's columns
+    const int row_local = lg * 32 + lane;
+    const uint32_t swz = static_cast<uint32_t>(row_local & 7);
+    uint8_t* obuf = smem + OFF_OUT + grp * OUT_BYTES;
+    uint8_t* orow = obuf + row_local * 128;
+    const bool issuer = (e & 3) == 0 && lane == 0;
+    const int bar_id = 1 + grp;
     uint32_t tile = 0;
     bool ok = true;
     int prob, v;
     for (int i = 0; ok && gemm_unit_at(p, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
       const GemmProblem& g = p.pr[prob];
       const GemmUnit u = gemm_decode(g, v);
-      const int n0 = u.n0;
+      const CUtensorMap* to = prob ? &tmap_o1 : &tmap_o0;
       const int m0 = u.m0 + static_cast<int>(rank) * BM;
-      const int out_mode = g.out_mode;
-      const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
-      if (!(ok = mbar_wait(tfull0 + 8 * buf, tph, abort_flag))) break;
+      const bool rows_inside = m0 < g.M;          // else this CTA's 128 rows lie beyond M: nothing to store
+      const int gcols = (BNS / 2) * u.ns;         // accumulator columns this group drains
+      const int c0 = grp * gcols;                 // the first of them
+      const int step = g.out_f32 ? 32 : 64;       // columns per staged sub-tile (128 bytes of output)
+      // sub-tiles of this group that lie inside N (uniform over the group)
+      int nsteps = (g.N - (u.n0 + c0) + step - 1) / step;
+      nsteps = nsteps < 0 ? 0 : (nsteps > gcols / step ? gcols / step : nsteps);
+      ok = __all_sync(0xffffffffu, mbar_wait(tfull, tile & 1, abort_flag));
+      if (!ok) break;
       tc_fence_after_sync();
-      const int row = m0 + lg * 32 + lane;
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN;
-#pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int col0 = n0 + c * 32;
-        if (col0 >= g.N) break;  // uniform over the warp
-        uint32_t r[32];
-        tmem_ld32(taddr + c * 32, r);
-        tmem_ld_wait();
-        if (row < g.M) {
-          const bool full_chunk = (col0 + 32 <= g.N);
-          if (out_mode == kOutStoreBF16 || out_mode == kOutAddBF16) {
-            __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(g.out) + row * g.ldo + col0;
-            if (full_chunk) {
-              uint4* o4 = reinterpret_cast<uint4*>(o);
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + c0;
+      if (nsteps == 0) {
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(tempty_leader);
+      }
+      for (int j = 0; j < nsteps; ++j) {
+        uint32_t w[32];  // 128 bytes of this thread's output row
+        if (g.out_f32) {
+          tmem_ld32(taddr + j * 32, w);
+          tmem_ld_wait();
+        } else {
+          uint32_t r0[32], r1[32];
+          tmem_ld32(taddr + j * 64, r0);
+          tmem_ld32(taddr + j * 64 + 32, r1);
+          tmem_ld_wait();
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                float x[8];
-#pragma unroll
-                for (int q = 0; q < 8; ++q) x[q] = __uint_as_float(r[8 * j + q]);
-                if (out_mode == kOutAddBF16) {
-                  const uint4 old = o4[j];
-                  x[0] += bf16_lo(old.x); x[1] += bf16_hi(old.x);
-                  x[2] += bf16_lo(old.y); x[3] += bf16_hi(old.y);
-                  x[4] += bf16_lo(old.z); x[5] += bf16_hi(old.z);
-                  x[6] += bf16_lo(old.w); x[7] += bf16_hi(old.w);
-                }
-                uint4 w;
-                w.x = pack_bf16x2(x[0], x[1]);
-                w.y = pack_bf16x2(x[2], x[3]);
-                w.z = pack_bf16x2(x[4], x[5]);
-                w.w = pack_bf16x2(x[6], x[7]);
-                o4[j] = w;
-              }
-            } else {
-              for (int j = 0; j < 32 && col0 + j < g.N; ++j) {
-                float x = __uint_as_float(r[j]);
-                if (out_mode == kOutAddBF16) x += __bfloat162float(o[j]);
-                o[j] = __float2bfloat16_rn(x);
-              }
-            }
-          } else {
-            float* o = reinterpret_cast<float*>(g.out) + row * g.ldo + col0;
-            if (out_mode == kOutAtomicF32) {
-              if (full_chunk) {
-#pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + j),
-                               "f"(__uint_as_float(r[j])), "f"(__uint_as_float(r[j + 1])),
-                               "f"(__uint_as_float(r[j + 2])), "f"(__uint_as_float(r[j + 3]))
-                               : "memory");
-              } else {
-                for (int j = 0; j < 32 && col0 + j < g.N; ++j) atomicAdd(o + j, __uint_as_float(r[j]));
-              }
-            } else if (full_chunk) {
-              float4* o4 = reinterpret_cast<float4*>(o);
-#pragma unroll
-              for (int j = 0; j < 8; ++j) {
-                float4 x = make_float4(__uint_as_float(r[4 * j]), __uint_as_float(r[4 * j + 1]),
-                                       __uint_as_float(r[4 * j + 2]), __uint_as_float(r[4 * j + 3]));
-                if (out_mode == kOutAddF32) {
-                  const float4 old = o4[j];
-                  x.x += old.x; x.y += old.y; x.z += old.z; x.w += old.w;
-                }
-                o4[j] = x;
-              }
-            } else {
-              for (int j = 0; j < 32 && col0 + j < g.N; ++j) {
-                float x = __uint_as_float(r[j]);
-                if (out_mode == kOutAddF32) x += o[j];
-                o[j] = x;
-              }
-            }
+          for (int q = 0; q < 16; ++q) {
+            w[q] = pack_bf16x2(__uint_as_float(r0[2 * q]), __uint_as_float(r0[2 * q + 1]));
+            w[16 + q] = pack_bf16x2(__uint_as_float(r1[2 * q]), __uint_as_float(r1[2 * q + 1]));
           }
         }
+        if (j == nsteps - 1) {
+          // everything this warp needs from tensor memory is in registers: release the accumulators
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(tempty_leader);
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          *reinterpret_cast<uint4*>(orow + ((static_cast<uint32_t>(q) ^ swz) << 4)) =
+              make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+        fence_proxy_async_smem();
+        named_barrier_sync(bar_id, 128);
+        if (issuer && rows_inside) {
+          const int col = u.n0 + c0 + j * step;
+          if (g.out_reduce)
+            tma_reduce_add_2d(to, smem_u32(obuf), col, m0);
+          else
+            tma_store_2d(to, smem_u32(obuf), col, m0);
+          tma_store_commit();
+          tma_store_wait_read<0>();  // the staging buffer may be overwritten after this
+        }
+        named_barrier_sync(bar_id, 128);
       }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);
     }
+    if (issuer) tma_store_wait_all<0>();
   }
 
   // ------------------------------ teardown ------------------------------------

@@ -38,19 +38,20 @@ PFN_cuTensorMapEncodeTiled_v12000 tensor_map_encoder() {
   return fn;
 }
 
-// 2-D bf16 tensor map with 128-byte swizzle.  inner = contiguous extent (elements),
-// outer = rows, ld = row stride (elements), box = {box_inner (64), box_outer}.
+// 2-D tensor map with 128-byte swizzle.  inner = contiguous extent (elements), outer = rows,
+// ld = row stride (elements), box = {box_inner (128 bytes' worth), box_outer}.
 bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t ld,
-              uint32_t box_inner, uint32_t box_outer) {
+              uint32_t box_inner, uint32_t box_outer, bool f32 = false) {
   auto enc = tensor_map_encoder();
   if (enc == nullptr) return false;
   cuuint64_t dims[2] = {inner, outer};
-  cuuint64_t strides[1] = {ld * 2};
+  cuuint64_t strides[1] = {ld * (f32 ? 4 : 2)};
   cuuint32_t box[2] = {box_inner, box_outer};
   cuuint32_t estr[2] = {1, 1};
-  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
-             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+             const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 struct DeviceInfo {
@@ -188,6 +189,8 @@ struct GemmOperands {
   long long lda;
   const void* B;
   long long ldb;
+  void* out;
+  long long ldo;
 };
 
 // k-steps one unit of a problem runs (its cost in the schedule)
@@ -203,16 +206,19 @@ int gemm_units(const GemmProblem& g) {
 int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, int* status, int sms,
                 cudaStream_t st) {
   using namespace gemm_cfg;
-  CUtensorMap maps[4];
+  CUtensorMap maps[6];
   GemmParams gp{};
   for (int i = 0; i < 2; ++i) {
     const int j = i < nprob ? i : 0;  // an unused slot repeats problem 0's (valid) maps
     const GemmProblem& g = pr[j];
-    const bool oka = g.a_mn ? make_map(&maps[2 * i], ops[j].A, g.M, g.K, ops[j].lda, 64, 64)
-                            : make_map(&maps[2 * i], ops[j].A, g.K, g.M, ops[j].lda, 64, BM);
-    const bool okb = g.b_mn ? make_map(&maps[2 * i + 1], ops[j].B, g.N, g.K, ops[j].ldb, 64, 64)
-                            : make_map(&maps[2 * i + 1], ops[j].B, g.K, g.N, ops[j].ldb, 64, BNH);
-    if (!oka || !okb) return NPD_ECUDA;
+    const bool oka = g.a_mn ? make_map(&maps[3 * i], ops[j].A, g.M, g.K, ops[j].lda, 64, 64)
+                            : make_map(&maps[3 * i], ops[j].A, g.K, g.M, ops[j].lda, 64, BM);
+    const bool okb = g.b_mn ? make_map(&maps[3 * i + 1], ops[j].B, g.N, g.K, ops[j].ldb, 64, 64)
+                            : make_map(&maps[3 * i + 1], ops[j].B, g.K, g.N, ops[j].ldb, 64, BNS / 2);
+    // output sub-tiles: 128 rows x 128 bytes
+    const bool oko = make_map(&maps[3 * i + 2], ops[j].out, g.N, g.M, ops[j].ldo, g.out_f32 ? 32 : 64, BM,
+                              g.out_f32 != 0);
+    if (!oka || !okb || !oko) return NPD_ECUDA;
     gp.pr[i] = g;
     gp.units[i] = i < nprob ? gemm_units(g) : 0;
   }
@@ -226,7 +232,8 @@ int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, int* 
   }
   gp.status = status;
   if (set_smem(gemm_bf16_kernel, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
-  gemm_bf16_kernel<<<2 * pairs, THREADS, SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], gp);
+  gemm_bf16_kernel<<<2 * pairs, THREADS, SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4],
+                                                          maps[5], gp);
   ++g_launches;
   return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
 }
@@ -402,34 +409,31 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     pr[0].a_mn = 1;
     pr[0].b_mn = 1;
     pr[0].k_splits = 1;
-    pr[0].ldo = a->ldw;
-    if (a->d_weight_dtype == NPD_DTYPE_F32) {
-      pr[0].out = static_cast<float*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw;
-      pr[0].out_mode = (a->flags & NPD_KD_ACCUMULATE_DW) ? kOutAddF32 : kOutStoreF32;
-    } else {
-      pr[0].out = static_cast<__nv_bfloat16*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw;
-      pr[0].out_mode = kOutStoreBF16;
-    }
-    ops[0] = {gbuf, ldg, a->hidden, a->ldh};
+    pr[0].out_f32 = a->d_weight_dtype == NPD_DTYPE_F32;
+    pr[0].out_reduce = (a->flags & NPD_KD_ACCUMULATE_DW) ? 1 : 0;
+    void* dw_rows = pr[0].out_f32
+                        ? static_cast<void*>(static_cast<float*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw)
+                        : static_cast<void*>(static_cast<__nv_bfloat16*>(a->d_weight) +
+                                             static_cast<size_t>(col0) * a->ldw);
+    ops[0] = {gbuf, ldg, a->hidden, a->ldh, dw_rows, a->ldw};
     // dH (+)= G_chunk W[col0 .. col0+cols)      (M = T, N = d, K = vocabulary rows of the chunk)
     pr[1].M = a->T;
     pr[1].N = a->d;
     pr[1].K = cols;
     pr[1].a_mn = 0;
     pr[1].b_mn = 1;
+    const __nv_bfloat16* w_rows = static_cast<const __nv_bfloat16*>(a->weight) + static_cast<size_t>(col0) * a->ldw;
     if (pl.dh_direct) {
       pr[1].k_splits = 1;
-      pr[1].out = a->d_hidden;
-      pr[1].ldo = a->ldh;
-      pr[1].out_mode = kOutStoreBF16;
+      pr[1].out_f32 = 0;
+      pr[1].out_reduce = 0;
+      ops[1] = {gbuf, ldg, w_rows, a->ldw, a->d_hidden, a->ldh};
     } else {
       pr[1].k_splits = std::max(1, std::min(pl.dh_ksplits, (cols + 63) / 64));
-      pr[1].out = dh_acc;
-      pr[1].ldo = a->d;
-      pr[1].out_mode = kOutAtomicF32;
+      pr[1].out_f32 = 1;
+      pr[1].out_reduce = 1;
+      ops[1] = {gbuf, ldg, w_rows, a->ldw, dh_acc, a->d};
     }
-    ops[1] = {gbuf, ldg, static_cast<const __nv_bfloat16*>(a->weight) + static_cast<size_t>(col0) * a->ldw,
-              a->ldw};
     if ((rc = launch_gemm(2, pr, ops, status, di.sms, st)) != NPD_OK) return rc;
     rec.mark();
   }
@@ -598,9 +602,10 @@ int npd_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, i
                   const void* B, int64_t ldb, int32_t b_mn_major, void* out, int64_t ldo,
                   int32_t out_mode, int32_t k_splits, void* cuda_stream) {
   if (M < 1 || N < 1 || K < 1 || A == nullptr || B == nullptr || out == nullptr) return NPD_EINVAL;
-  if (out_mode < kOutStoreF32 || out_mode > kOutAddBF16 || k_splits < 1) return NPD_EINVAL;
-  if (k_splits > 1 && out_mode != kOutAtomicF32) return NPD_EINVAL;
-  if (!aligned16(A) || !aligned16(B) || !aligned16(out) || (lda % 8) || (ldb % 8) || (ldo % 8))
+  if (out_mode < NPD_GEMM_STORE_F32 || out_mode > NPD_GEMM_ATOMIC_F32 || k_splits < 1) return NPD_EINVAL;
+  if (k_splits > 1 && out_mode != NPD_GEMM_ATOMIC_F32 && out_mode != NPD_GEMM_ADD_F32) return NPD_EINVAL;
+  const bool f32 = out_mode != NPD_GEMM_STORE_BF16;
+  if (!aligned16(A) || !aligned16(B) || !aligned16(out) || (lda % 8) || (ldb % 8) || (ldo % (f32 ? 4 : 8)))
     return NPD_EALIGN;
   if (lda < (a_mn_major ? M : K) || ldb < (b_mn_major ? N : K) || ldo < N) return NPD_ESHAPE;
   DeviceInfo di;
@@ -614,10 +619,9 @@ int npd_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, i
   pr.a_mn = a_mn_major != 0;
   pr.b_mn = b_mn_major != 0;
   pr.k_splits = k_splits;
-  pr.out = out;
-  pr.ldo = ldo;
-  pr.out_mode = out_mode;
-  const GemmOperands ops{A, lda, B, ldb};
+  pr.out_f32 = f32;
+  pr.out_reduce = out_mode == NPD_GEMM_ADD_F32 || out_mode == NPD_GEMM_ATOMIC_F32;
+  const GemmOperands ops{A, lda, B, ldb, out, ldo};
   return launch_gemm(1, &pr, &ops, nullptr, di.sms, static_cast<cudaStream_t>(cuda_stream));
 }
 

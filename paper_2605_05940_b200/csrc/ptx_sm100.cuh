@@ -102,6 +102,15 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, uint32_t src_
       "r"(src_smem), "r"(x), "r"(y)
       : "memory");
 }
+// Same, but the tile is ADDED to global memory (element-wise atomic add in the map's data type).
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* m, uint32_t src_smem, int32_t x,
+                                                  int32_t y) {
+  asm volatile(
+      "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+          reinterpret_cast<uint64_t>(m)),
+      "r"(src_smem), "r"(x), "r"(y)
+      : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() {
   asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
