@@ -39,14 +39,27 @@ struct GemmProblem {
   int k_splits;    // > 1 only with out_reduce
   int out_f32;     // output elements: 1 = fp32, 0 = bf16
   int out_reduce;  // 1 = D += acc (atomic, any number of adders), 0 = D = acc
+  // Row-block indirection for the backward over the 128-row blocks of a packed batch that hold
+  // loss tokens (blocks[i] = first row of block i, nblocks[0] = how many; both on the device):
+  int dyn_m;       // M = 128 * nblocks[0]: A's rows are the listed blocks, stored back to back
+  int dyn_k;       // K = 128 * nblocks[0]: A's k-extent likewise
+  int map_bk;      // B's k coordinate of compact k-row i*128+j is blocks[i]+j
+  int map_om;      // output row of compact row i*128+j is blocks[i]+j
 };
 
 struct GemmParams {
   GemmProblem pr[2];
+  int nprob;           // 1 or 2
+  const int* nblocks;  // device; read only when a problem has dyn_m / dyn_k
+  const int* blocks;   // device; read only when a problem has map_bk / map_om
+  int* status;         // device status word
+};
+
+// How the units of the one or two problems are dealt to the CTA pairs.
+struct GemmSched {
   int units[2];    // work units of each problem (tiles x k_splits); units[1] = 0 for a single problem
   int q0, rem0;    // units[0] = q0 * pairs + rem0
   int extra1;      // units of problem 1 that each pair WITHOUT a remainder unit of problem 0 takes first
-  int* status;     // device status word
 };
 
 namespace gemm_cfg {
@@ -72,7 +85,7 @@ constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;  // + barriers + alignment
 // The i-th unit of CTA pair c out of C.  Problem-0 units go round robin.  The pairs that got
 // one unit fewer of problem 0 (c >= rem0) make up for it with `extra1` units of problem 1;
 // the rest of problem 1 goes round robin over all pairs.
-__host__ __device__ inline bool gemm_unit_at(const GemmParams& p, int c, int C, int i, int& prob, int& v) {
+__host__ __device__ inline bool gemm_unit_at(const GemmSched& p, int c, int C, int i, int& prob, int& v) {
   const int n0 = p.q0 + (c < p.rem0 ? 1 : 0);
   if (i < n0) {
     prob = 0;
@@ -95,6 +108,32 @@ __host__ __device__ inline bool gemm_unit_at(const GemmParams& p, int c, int C, 
   }
   v = base + j * C + c;
   return v < p.units[1];
+}
+
+__host__ __device__ inline int gemm_unit_ksteps(const GemmProblem& g) {
+  const int kt = (g.K + 63) / 64;
+  const int per = (kt + g.k_splits - 1) / g.k_splits;
+  return per > 0 ? per : 1;
+}
+// Resolves the device-side dimensions and deals the units to C pairs.
+__device__ __forceinline__ void gemm_setup(const GemmParams& p, int C, GemmProblem (&pr)[2], GemmSched& sc) {
+  pr[0] = p.pr[0];
+  pr[1] = p.pr[1];
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    if (pr[i].dyn_m) pr[i].M = 128 * __ldg(p.nblocks);
+    if (pr[i].dyn_k) pr[i].K = 128 * __ldg(p.nblocks);
+    const int tiles = ((pr[i].M + 255) / 256) * ((pr[i].N + 511) / 512);
+    sc.units[i] = i < p.nprob ? tiles * pr[i].k_splits : 0;
+  }
+  sc.q0 = sc.units[0] / C;
+  sc.rem0 = sc.units[0] % C;
+  sc.extra1 = 0;
+  if (sc.units[1] > 0 && sc.rem0 > 0) {
+    const int c0 = gemm_unit_ksteps(pr[0]), c1 = gemm_unit_ksteps(pr[1]);
+    const int want = (c0 + c1 / 2) / c1, can = sc.units[1] / (C - sc.rem0);
+    sc.extra1 = want < can ? want : can;
+  }
 }
 
 struct GemmUnit {
@@ -150,7 +189,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
     prefetch_tmap(&tmap_a0);
     prefetch_tmap(&tmap_b0);
     prefetch_tmap(&tmap_o0);
-    if (p.units[1] > 0) {
+    if (p.nprob > 1) {
       prefetch_tmap(&tmap_a1);
       prefetch_tmap(&tmap_b1);
       prefetch_tmap(&tmap_o1);
@@ -165,14 +204,19 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
   const uint32_t full_leader = mapa_shared(full0, 0);
   const uint32_t tempty_leader = mapa_shared(tempty, 0);
 
+  // every role resolves the same problems and the same deal of units
+  GemmProblem pr[2];
+  GemmSched sc;
+  gemm_setup(p, num_clusters, pr, sc);
+
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
       int prob, v;
-      for (int i = 0; ok && gemm_unit_at(p, cluster_id, num_clusters, i, prob, v); ++i) {
-        const GemmProblem& g = p.pr[prob];
+      for (int i = 0; ok && gemm_unit_at(sc, cluster_id, num_clusters, i, prob, v); ++i) {
+        const GemmProblem& g = prob ? pr[1] : pr[0];
         const GemmUnit u = gemm_decode(g, v);
         const CUtensorMap* ta = prob ? &tmap_a1 : &tmap_a0;
         const CUtensorMap* tb = prob ? &tmap_b1 : &tmap_b0;
@@ -187,6 +231,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
           const uint32_t fb = full_leader + 8 * s;
           const uint32_t sa = smem_u32(smem_a + s * A_BYTES), sb = smem_u32(smem_b + s * B_BYTES);
           const int k0 = kt * BK;
+          // B's k rows: straight, or the rows of the kt/2-th listed block
+          const int kb = g.map_bk ? __ldg(p.blocks + (kt >> 1)) + (kt & 1) * BK : k0;
           if (g.a_mn) {
 #pragma unroll
             for (int j = 0; j < BM / 64; ++j) tma_load_2d_pair(sa + j * 8192, ta, fb, m0 + 64 * j, k0);
@@ -198,9 +244,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
             const int nh = n0 + h * BNS;
             if (g.b_mn) {
 #pragma unroll
-              for (int j = 0; j < BNS / 2 / 64; ++j) tma_load_2d_pair(sbh + j * 8192, tb, fb, nh + 64 * j, k0);
+              for (int j = 0; j < BNS / 2 / 64; ++j) tma_load_2d_pair(sbh + j * 8192, tb, fb, nh + 64 * j, kb);
             } else {
-              tma_load_2d_pair(sbh, tb, fb, k0, nh);
+              tma_load_2d_pair(sbh, tb, fb, kb, nh);
             }
           }
         }
@@ -219,8 +265,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
       uint32_t it = 0, tile = 0;
       bool ok = true;
       int prob, v;
-      for (int i = 0; ok && gemm_unit_at(p, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
-        const GemmProblem& g = p.pr[prob];
+      for (int i = 0; ok && gemm_unit_at(sc, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
+        const GemmProblem& g = prob ? pr[1] : pr[0];
         const GemmUnit u = gemm_decode(g, v);
         const uint32_t idesc = umma_idesc_bf16(PM, BNS, g.a_mn != 0, g.b_mn != 0);
         // the accumulators are free once every epilogue warp of the pair has read the last tile
@@ -262,12 +308,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
     uint32_t tile = 0;
     bool ok = true;
     int prob, v;
-    for (int i = 0; ok && gemm_unit_at(p, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
-      const GemmProblem& g = p.pr[prob];
+    for (int i = 0; ok && gemm_unit_at(sc, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
+      const GemmProblem& g = prob ? pr[1] : pr[0];
       const GemmUnit u = gemm_decode(g, v);
       const CUtensorMap* to = prob ? &tmap_o1 : &tmap_o0;
       const int m0 = u.m0 + static_cast<int>(rank) * BM;
       const bool rows_inside = m0 < g.M;          // else this CTA's 128 rows lie beyond M: nothing to store
+      // output rows: straight, or the rows of the listed block
+      const int out_row0 = (g.map_om && rows_inside) ? __ldg(p.blocks + (m0 >> 7)) : m0;
+      const bool no_k = u.kt0 == u.kt1;           // empty k range: the accumulators hold nothing, D = 0
       const int gcols = (BNS / 2) * u.ns;         // accumulator columns this group drains
       const int c0 = grp * gcols;                 // the first of them
       const int step = g.out_f32 ? 32 : 64;       // columns per staged sub-tile (128 bytes of output)
@@ -285,7 +334,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
       }
       for (int j = 0; j < nsteps; ++j) {
         uint32_t w[32];  // 128 bytes of this thread's output row
-        if (g.out_f32) {
+        if (no_k) {
+#pragma unroll
+          for (int q = 0; q < 32; ++q) w[q] = 0u;
+        } else if (g.out_f32) {
           tmem_ld32(taddr + j * 32, w);
           tmem_ld_wait();
         } else {
@@ -314,9 +366,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
         if (issuer && rows_inside) {
           const int col = u.n0 + c0 + j * step;
           if (g.out_reduce)
-            tma_reduce_add_2d(to, smem_u32(obuf), col, m0);
+            tma_reduce_add_2d(to, smem_u32(obuf), col, out_row0);
           else
-            tma_store_2d(to, smem_u32(obuf), col, m0);
+            tma_store_2d(to, smem_u32(obuf), col, out_row0);
           tma_store_commit();
           tma_store_wait_read<0>();  // the staging buffer may be overwritten after this
         }

@@ -45,11 +45,12 @@ enum : int { kPMaxA = 0, kPSumA, kPCross, kPMaxB, kPSumB, kPSumA1, kPSumB1, kPFi
 struct KdTileParams {
   int T, V;
   int ksteps;       // d / 64
-  int row_blocks;   // ceil(T / 128)
-  int row_pairs;    // ceil(T / 256): one pair of CTAs owns 256 token rows
+  const int* plan;  // {128-row blocks that hold loss tokens, pairs of them, forward runs, 0} (device)
+  const int* list;  // first packed row of every such block, in order; a pair of CTAs owns two
+                    // consecutive entries
   int vt_begin;     // first 256-wide vocabulary tile of this launch
-  int vt_count;     // number of vocabulary tiles of this launch
-  int nsplit;       // the vt_count tiles are cut into nsplit runs; a unit = (row pair, run)
+  int vt_count;     // number of vocabulary tiles of this launch; they are cut into runs (forward:
+                    // plan[2] runs, gradient: one tile per run); a unit = (pair of blocks, run)
   float scale2;     // log2(e) / tau
   float tau;
   // forward
@@ -58,7 +59,8 @@ struct KdTileParams {
   const float* lse2_a;  // [T] log2-sum-exp2 of the scaled teacher logits
   const float* lse2_b;  // [T] same for the student
   const float* coef;    // [T] grad_scale * m_t / tau
-  int g_col0;           // vocabulary column that scratch column 0 holds
+  int g_col0;           // vocabulary column that scratch column 0 holds; scratch row = position in
+                        // the block list * 128 + row within the block
   int* status;
 };
 
@@ -140,13 +142,18 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   const uint32_t full_leader = mapa_shared(full0, 0);
   const uint32_t tempty_leader = mapa_shared(tempty0, 0);
 
-  const int units = p.row_pairs * p.nsplit;
-  // r = this CTA's 128-row block of the unit's row pair
-  auto run_of = [&](int u, int& r, int& s, int& vt0, int& vt1) {
-    r = 2 * (u % p.row_pairs) + static_cast<int>(rank);
-    s = u / p.row_pairs;
-    vt0 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * s / p.nsplit);
-    vt1 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * (s + 1) / p.nsplit);
+  const int nact = p.plan[0], pairs = p.plan[1];
+  const int nsplit = kMode == kForward ? p.plan[2] : p.vt_count;
+  const int units = pairs * nsplit;
+  // slot = this CTA's position in the block list, r = that block's first packed row, or -1
+  // when the list has an odd length and this CTA has no block (it then stages the rows from 0
+  // and writes nothing).
+  auto run_of = [&](int u, int& slot, int& r, int& s, int& vt0, int& vt1) {
+    slot = 2 * (u % pairs) + static_cast<int>(rank);
+    r = slot < nact ? __ldg(p.list + slot) : -1;
+    s = u / pairs;
+    vt0 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * s / nsplit);
+    vt1 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * (s + 1) / nsplit);
   };
 
   if (warp == 0) {
@@ -155,8 +162,9 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       uint32_t it = 0;
       bool ok = true;
       for (int u = cluster_id; u < units && ok; u += num_clusters) {
-        int r, s, vt0, vt1;
-        run_of(u, r, s, vt0, vt1);
+        int slot, r, s, vt0, vt1;
+        run_of(u, slot, r, s, vt0, vt1);
+        const int rl = r < 0 ? 0 : r;
         for (int vt = vt0; vt < vt1 && ok; ++vt) {
           for (int ks = 0; ks < p.ksteps; ++ks, ++it) {
             const uint32_t st = it % STAGES, ph = (it / STAGES) & 1;
@@ -164,7 +172,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             // the leader's barrier counts the bytes of both CTAs' loads of this stage
             if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, 2 * (A_BYTES + B_BYTES));
             const uint32_t fb = full_leader + 8 * st;
-            tma_load_2d_pair(smem_u32(smem + OFF_A + st * A_BYTES), &tmap_h, fb, ks * BK, r * BM);
+            tma_load_2d_pair(smem_u32(smem + OFF_A + st * A_BYTES), &tmap_h, fb, ks * BK, rl);
             tma_load_2d_pair(smem_u32(smem + OFF_B + st * B_BYTES), &tmap_w, fb, ks * BK,
                              vt * BN + static_cast<int>(rank) * BNH);
           }
@@ -185,8 +193,9 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       uint32_t it = 0, tile = 0;
       bool ok = true;
       for (int u = cluster_id; u < units && ok; u += num_clusters) {
-        int r, s, vt0, vt1;
-        run_of(u, r, s, vt0, vt1);
+        int slot, r, s, vt0, vt1;
+        run_of(u, slot, r, s, vt0, vt1);
+        (void)slot;
         for (int vt = vt0; vt < vt1 && ok; ++vt, ++tile) {
           const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
           if (!(ok = mbar_wait(tempty0 + 8 * buf, tph ^ 1, abort_flag))) break;
@@ -216,8 +225,9 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       uint32_t zit = 0;  // sub-tile pairs issued; both halves advance together
       bool ok = true;
       for (int u = cluster_id; u < units && ok; u += num_clusters) {
-        int r, s, vt0, vt1;
-        run_of(u, r, s, vt0, vt1);
+        int slot, r, s, vt0, vt1;
+        run_of(u, slot, r, s, vt0, vt1);
+        const int rl = r < 0 ? 0 : r;
         for (int vt = vt0; vt < vt1 && ok; ++vt) {
           for (int j = 0; j < BN / 2 / ZSUB_COLS && ok; ++j, ++zit) {
             const uint32_t q = zit % ZQ, ph = (zit / ZQ) & 1;
@@ -227,7 +237,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
               if (!(ok = mbar_wait(zempty0 + bi, ph ^ 1, abort_flag))) break;
               mbar_arrive_expect_tx(zfull0 + bi, ZSUB_BYTES);
               tma_load_2d(smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES), &tmap_t, zfull0 + bi,
-                          col, r * BM);
+                          col, rl);
             }
           }
         }
@@ -249,12 +259,13 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     uint32_t tile = 0, zit = 0;
     bool ok = true;
     for (int u = cluster_id; u < units && ok; u += num_clusters) {
-      int r, s, vt0, vt1;
-      run_of(u, r, s, vt0, vt1);
-      const int row = r * BM + row_local;
+      int slot, r, s, vt0, vt1;
+      run_of(u, slot, r, s, vt0, vt1);
+      const int row = r < 0 ? p.T : r + row_local;  // token row; >= T: nothing to read or write
       // forward state (base-2 domain): running max / sum of the scaled teacher (a) and student (b)
       float m_a = -INFINITY, s_a = 0.f, cross = 0.f, m_b = -INFINITY, s_b = 0.f, s_a1 = 0.f, s_b1 = 0.f;
-      float g_lse_a = 0.f, g_lse_b = 0.f, g_coef = 0.f;
+      // rows without a token (beyond T, or a CTA without a block): probabilities 0, gradient 0
+      float g_lse_a = 1e30f, g_lse_b = 1e30f, g_coef = 0.f;
       if (kMode == kGradient && row < p.T) {
         g_lse_a = p.lse2_a[row];
         g_lse_b = p.lse2_b[row];
@@ -363,9 +374,9 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             fence_proxy_async_smem();
             named_barrier_sync(1 + half, 128);
             if (lg == 0 && lane == 0) {
-              if (r * BM < p.T) {
+              if (r >= 0) {
                 tma_store_2d(&tmap_g, smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES),
-                             sub_col0 - p.g_col0, r * BM);
+                             sub_col0 - p.g_col0, slot * BM);
                 tma_store_commit();
                 tma_store_wait_read<0>();
               }

@@ -67,40 +67,24 @@ int device_info(DeviceInfo* out) {
   return NPD_OK;
 }
 
-// How many runs to cut the vocabulary tiles into so that row_pairs * nsplit work
-// units spread evenly over the CTA pairs.  Cost = rounds of units x tiles per unit.
-int choose_nsplit(int row_blocks, int vtiles, int sms) {
-  int best = 1;
-  long long best_cost = -1;
-  const int max_split = std::min(vtiles, 128);
-  for (int ns = 1; ns <= max_split; ++ns) {
-    const long long rounds = (static_cast<long long>(row_blocks) * ns + sms - 1) / sms;
-    const long long per = (vtiles + ns - 1) / ns;
-    const long long cost = rounds * per * 64 + ns;  // small bias towards fewer splits
-    if (best_cost < 0 || cost < best_cost) {
-      best_cost = cost;
-      best = ns;
-    }
-  }
-  return best;
-}
-
 struct Plan {
-  int row_blocks, row_pairs, vtiles, nsplit, nslots;
+  int row_blocks, vtiles, clusters;
+  int nsplit_max;     // upper bound of the forward's vocabulary runs (the device picks the number)
   int chunk_cols;     // vocabulary columns per gradient chunk (multiple of 256)
   int nchunks;
   int dh_ksplits;     // split-K of the dH product of a full chunk
   bool dh_direct;     // dH stored straight to the output (one chunk, no split-K); else fp32 atomics
   bool grads;
-  size_t off_status, off_partials, off_lse_a, off_lse_b, off_coef, off_g, off_dh, total;
+  size_t off_status, off_plan, off_list, off_partials, off_lse_a, off_lse_b, off_coef, off_g, off_dh, total;
 };
 
 int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   pl->row_blocks = (a->T + 127) / 128;
-  pl->row_pairs = (a->T + 255) / 256;
   pl->vtiles = (a->V + 255) / 256;
-  pl->nsplit = choose_nsplit(pl->row_pairs, pl->vtiles, std::max(sms / 2, 1));
-  pl->nslots = 2 * pl->nsplit;
+  pl->clusters = std::max(sms / 2, 1);
+  // The fewer row pairs there are, the more runs are needed to fill the CTA pairs.
+  const int row_pairs = (pl->row_blocks + 1) / 2;
+  pl->nsplit_max = std::min(pl->vtiles, std::max(4, std::min(64, 8 * pl->clusters / row_pairs)));
   pl->grads = a->d_hidden != nullptr || a->d_weight != nullptr;
   // Vocabulary chunks of the backward: the bf16 logit-gradient block [T, chunk_cols] is the only
   // thing that travels between the gradient tiles and the two contractions.  Default: the
@@ -123,8 +107,12 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   size_t off = 0;
   pl->off_status = off;
   off += 1024;
+  pl->off_plan = off;
+  off += 1024;
+  pl->off_list = off;
+  off = align_up(off + sizeof(int) * static_cast<size_t>(pl->row_blocks), 1024);
   pl->off_partials = off;
-  off = align_up(off + sizeof(float) * pl->nslots * kPFields * static_cast<size_t>(a->T), 1024);
+  off = align_up(off + sizeof(float) * 2 * pl->nsplit_max * kPFields * static_cast<size_t>(a->T), 1024);
   pl->off_lse_a = off;
   off = align_up(off + sizeof(float) * a->T, 1024);
   pl->off_lse_b = off;
@@ -134,7 +122,7 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   pl->off_g = off;
   pl->off_dh = off;
   if (pl->grads) {
-    off = align_up(off + 2 * static_cast<size_t>(a->T) * cc, 1024);
+    off = align_up(off + 2 * static_cast<size_t>(pl->row_blocks) * 128 * cc, 1024);
     pl->off_dh = off;
     if (!pl->dh_direct) off = align_up(off + sizeof(float) * static_cast<size_t>(a->T) * a->d, 1024);
   }
@@ -191,46 +179,42 @@ struct GemmOperands {
   long long ldb;
   void* out;
   long long ldo;
+  long long b_rows;    // rows of B's / the output's memory when they are addressed through the
+  long long out_rows;  // block list (else unused)
 };
 
-// k-steps one unit of a problem runs (its cost in the schedule)
-int gemm_unit_ksteps(const GemmProblem& g) {
-  return std::max(1, ((g.K + gemm_cfg::BK - 1) / gemm_cfg::BK + g.k_splits - 1) / g.k_splits);
-}
-int gemm_units(const GemmProblem& g) {
-  using namespace gemm_cfg;
-  return ((g.M + PM - 1) / PM) * ((g.N + BN - 1) / BN) * g.k_splits;
-}
-
 // One launch for one or two problems (see gemm_sm100.cuh for how the units are dealt).
-int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, int* status, int sms,
-                cudaStream_t st) {
+// a_rows / a_kext: extents of A's tensor map when M or K is only known on the device.
+int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const int* nblocks,
+                const int* blocks, int max_blocks, int* status, int sms, cudaStream_t st) {
   using namespace gemm_cfg;
   CUtensorMap maps[6];
   GemmParams gp{};
+  long long units = 0;
   for (int i = 0; i < 2; ++i) {
     const int j = i < nprob ? i : 0;  // an unused slot repeats problem 0's (valid) maps
     const GemmProblem& g = pr[j];
-    const bool oka = g.a_mn ? make_map(&maps[3 * i], ops[j].A, g.M, g.K, ops[j].lda, 64, 64)
-                            : make_map(&maps[3 * i], ops[j].A, g.K, g.M, ops[j].lda, 64, BM);
-    const bool okb = g.b_mn ? make_map(&maps[3 * i + 1], ops[j].B, g.N, g.K, ops[j].ldb, 64, 64)
-                            : make_map(&maps[3 * i + 1], ops[j].B, g.K, g.N, ops[j].ldb, 64, BNS / 2);
+    // extents as the maps see them: device-side dimensions take their upper bound
+    const uint64_t am = g.dyn_m ? 128ull * max_blocks : g.M, ak = g.dyn_k ? 128ull * max_blocks : g.K;
+    const uint64_t bk = (g.dyn_k || g.map_bk) ? static_cast<uint64_t>(ops[j].b_rows) : g.K;
+    const uint64_t om = (g.dyn_m || g.map_om) ? static_cast<uint64_t>(ops[j].out_rows) : g.M;
+    const bool oka = g.a_mn ? make_map(&maps[3 * i], ops[j].A, am, ak, ops[j].lda, 64, 64)
+                            : make_map(&maps[3 * i], ops[j].A, ak, am, ops[j].lda, 64, BM);
+    const bool okb = g.b_mn ? make_map(&maps[3 * i + 1], ops[j].B, g.N, bk, ops[j].ldb, 64, 64)
+                            : make_map(&maps[3 * i + 1], ops[j].B, bk, g.N, ops[j].ldb, 64, BNS / 2);
     // output sub-tiles: 128 rows x 128 bytes
-    const bool oko = make_map(&maps[3 * i + 2], ops[j].out, g.N, g.M, ops[j].ldo, g.out_f32 ? 32 : 64, BM,
+    const bool oko = make_map(&maps[3 * i + 2], ops[j].out, g.N, om, ops[j].ldo, g.out_f32 ? 32 : 64, BM,
                               g.out_f32 != 0);
     if (!oka || !okb || !oko) return NPD_ECUDA;
     gp.pr[i] = g;
-    gp.units[i] = i < nprob ? gemm_units(g) : 0;
+    if (i < nprob)
+      units += static_cast<long long>((am + PM - 1) / PM) * ((g.N + BN - 1) / BN) * g.k_splits;
   }
-  const int pairs = std::max(1, std::min(gp.units[0] + gp.units[1], std::max(sms / 2, 1)));
-  gp.q0 = gp.units[0] / pairs;
-  gp.rem0 = gp.units[0] % pairs;
-  gp.extra1 = 0;
-  if (nprob == 2 && gp.rem0 > 0) {
-    const int c0 = gemm_unit_ksteps(pr[0]), c1 = gemm_unit_ksteps(pr[1]);
-    gp.extra1 = std::min((c0 + c1 / 2) / c1, gp.units[1] / (pairs - gp.rem0));
-  }
+  gp.nprob = nprob;
+  gp.nblocks = nblocks;
+  gp.blocks = blocks;
   gp.status = status;
+  const int pairs = static_cast<int>(std::max<long long>(1, std::min<long long>(units, std::max(sms / 2, 1))));
   if (set_smem(gemm_bf16_kernel, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
   gemm_bf16_kernel<<<2 * pairs, THREADS, SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4],
                                                           maps[5], gp);
@@ -244,8 +228,8 @@ int launch_kd_tile(bool tau_one, const CUtensorMap& mh, const CUtensorMap& mw, c
   using namespace kd_cfg;
   auto k = tau_one ? kd_tile_kernel<kMode, true> : kd_tile_kernel<kMode, false>;
   if (set_smem(k, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
-  const int units = kp.row_pairs * kp.nsplit;
-  const int grid = 2 * std::min(units, std::max(sms / 2, 1));  // CTA pairs
+  // the number of units is only known on the device: always one CTA pair per two SMs
+  const int grid = 2 * std::max(sms / 2, 1);
   k<<<grid, THREADS, SMEM_BYTES, st>>>(mh, mw, mt, mg, kp);
   ++g_launches;
   return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
@@ -300,6 +284,8 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   uint8_t* ws = static_cast<uint8_t*>(a->workspace);
   int* status = reinterpret_cast<int*>(ws + pl.off_status);
+  int* plan = reinterpret_cast<int*>(ws + pl.off_plan);
+  int* list = reinterpret_cast<int*>(ws + pl.off_list);
   float* partials = reinterpret_cast<float*>(ws + pl.off_partials);
   float* lse_a = reinterpret_cast<float*>(ws + pl.off_lse_a);
   float* lse_b = reinterpret_cast<float*>(ws + pl.off_lse_b);
@@ -324,17 +310,29 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     ++g_launches;
   }
 
+  // ---- cover the tokens with loss by 128-row blocks; everything below works on those only ----
+  {
+    const int words = (a->T + 31) / 32;
+    const int bitmap_words = words <= 48 * 1024 ? words : 0;  // up to 192 KB of shared memory
+    if (bitmap_words * 4 > 48 * 1024 &&
+        set_smem(plan_blocks_kernel, bitmap_words * 4) != NPD_OK)
+      return NPD_ECUDA;
+    plan_blocks_kernel<<<1, 1024, bitmap_words * 4, st>>>(a->T, a->loss_mask, bitmap_words, pl.vtiles,
+                                                          pl.nsplit_max, pl.clusters, plan, list);
+  }
+  ++g_launches;
+  if (cudaGetLastError() != cudaSuccess) return NPD_ECUDA;
+
   rec.mark();
-  // ---- forward: statistics per (row block, vocabulary run), then the per-token merge ----
+  // ---- forward: statistics per (pair of row blocks, vocabulary run), then the per-token merge ----
   KdTileParams kp{};
   kp.T = a->T;
   kp.V = a->V;
   kp.ksteps = a->d / 64;
-  kp.row_blocks = pl.row_blocks;
-  kp.row_pairs = pl.row_pairs;
+  kp.plan = plan;
+  kp.list = list;
   kp.vt_begin = 0;
   kp.vt_count = pl.vtiles;
-  kp.nsplit = pl.nsplit;
   kp.scale2 = scale2;
   kp.tau = a->temperature;
   kp.partials = partials;
@@ -346,7 +344,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   cp.T = a->T;
   cp.d = a->d;
   cp.V = a->V;
-  cp.nslots = pl.nslots;
+  cp.plan = plan;
   cp.partials = partials;
   cp.hidden = static_cast<const __nv_bfloat16*>(a->hidden);
   cp.weight = static_cast<const __nv_bfloat16*>(a->weight);
@@ -378,20 +376,26 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   __nv_bfloat16* gbuf = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_g);
   float* dh_acc = reinterpret_cast<float*>(ws + pl.off_dh);
   const long long ldg = pl.chunk_cols;
-  if (!pl.dh_direct &&
-      cudaMemsetAsync(dh_acc, 0, sizeof(float) * static_cast<size_t>(a->T) * a->d, st) != cudaSuccess)
+  // rows of blocks without loss are never written by the contractions: they start as zeros
+  if (pl.dh_direct) {
+    if (cudaMemset2DAsync(a->d_hidden, static_cast<size_t>(a->ldh) * 2, 0, static_cast<size_t>(a->d) * 2,
+                          a->T, st) != cudaSuccess)
+      return NPD_ECUDA;
+  } else if (cudaMemsetAsync(dh_acc, 0, sizeof(float) * static_cast<size_t>(a->T) * a->d, st) !=
+             cudaSuccess) {
     return NPD_ECUDA;
+  }
   for (int c = 0; c < pl.nchunks; ++c) {
     const int col0 = c * pl.chunk_cols;
     const int cols = std::min(pl.chunk_cols, a->V - col0);  // columns of this chunk inside V
     if (cols <= 0) break;
     const int cols_pad = std::min(pl.chunk_cols, pl.vtiles * 256 - col0);
     CUtensorMap mg;
-    if (!make_map(&mg, gbuf, cols_pad, a->T, ldg, 64, 128)) return NPD_ECUDA;
+    if (!make_map(&mg, gbuf, cols_pad, static_cast<uint64_t>(pl.row_blocks) * 128, ldg, 64, 128))
+      return NPD_ECUDA;
     KdTileParams gp = kp;
     gp.vt_begin = col0 / 256;
     gp.vt_count = cols_pad / 256;
-    gp.nsplit = gp.vt_count;
     gp.partials = nullptr;
     gp.lse2_a = lse_a;
     gp.lse2_b = lse_b;
@@ -402,10 +406,14 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
 
     GemmProblem pr[2] = {};
     GemmOperands ops[2] = {};
-    // dW[col0 .. col0+cols) = G_chunk^T H       (M = vocabulary rows, N = d, K = T)
+    // The logit-gradient block holds the active row blocks back to back (scratch row = position
+    // in the list * 128 + row within the block); H and dH are addressed through the list.
+    // dW[col0 .. col0+cols) = G_chunk^T H       (M = vocabulary rows, N = d, K = active token rows)
     pr[0].M = cols;
     pr[0].N = a->d;
-    pr[0].K = a->T;
+    pr[0].K = 0;
+    pr[0].dyn_k = 1;
+    pr[0].map_bk = 1;
     pr[0].a_mn = 1;
     pr[0].b_mn = 1;
     pr[0].k_splits = 1;
@@ -415,9 +423,11 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
                         ? static_cast<void*>(static_cast<float*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw)
                         : static_cast<void*>(static_cast<__nv_bfloat16*>(a->d_weight) +
                                              static_cast<size_t>(col0) * a->ldw);
-    ops[0] = {gbuf, ldg, a->hidden, a->ldh, dw_rows, a->ldw};
-    // dH (+)= G_chunk W[col0 .. col0+cols)      (M = T, N = d, K = vocabulary rows of the chunk)
-    pr[1].M = a->T;
+    ops[0] = {gbuf, ldg, a->hidden, a->ldh, dw_rows, a->ldw, a->T, 0};
+    // dH (+)= G_chunk W[col0 .. col0+cols)      (M = active token rows, N = d, K = the chunk's columns)
+    pr[1].M = 0;
+    pr[1].dyn_m = 1;
+    pr[1].map_om = 1;
     pr[1].N = a->d;
     pr[1].K = cols;
     pr[1].a_mn = 0;
@@ -427,14 +437,14 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
       pr[1].k_splits = 1;
       pr[1].out_f32 = 0;
       pr[1].out_reduce = 0;
-      ops[1] = {gbuf, ldg, w_rows, a->ldw, a->d_hidden, a->ldh};
+      ops[1] = {gbuf, ldg, w_rows, a->ldw, a->d_hidden, a->ldh, 0, a->T};
     } else {
       pr[1].k_splits = std::max(1, std::min(pl.dh_ksplits, (cols + 63) / 64));
       pr[1].out_f32 = 1;
       pr[1].out_reduce = 1;
-      ops[1] = {gbuf, ldg, w_rows, a->ldw, dh_acc, a->d};
+      ops[1] = {gbuf, ldg, w_rows, a->ldw, dh_acc, a->d, 0, a->T};
     }
-    if ((rc = launch_gemm(2, pr, ops, status, di.sms, st)) != NPD_OK) return rc;
+    if ((rc = launch_gemm(2, pr, ops, plan, list, pl.row_blocks, status, di.sms, st)) != NPD_OK) return rc;
     rec.mark();
   }
   if (!pl.dh_direct) {
@@ -621,8 +631,8 @@ int npd_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, i
   pr.k_splits = k_splits;
   pr.out_f32 = f32;
   pr.out_reduce = out_mode == NPD_GEMM_ADD_F32 || out_mode == NPD_GEMM_ATOMIC_F32;
-  const GemmOperands ops{A, lda, B, ldb, out, ldo};
-  return launch_gemm(1, &pr, &ops, nullptr, di.sms, static_cast<cudaStream_t>(cuda_stream));
+  const GemmOperands ops{A, lda, B, ldb, out, ldo, 0, 0};
+  return launch_gemm(1, &pr, &ops, nullptr, nullptr, 0, nullptr, di.sms, static_cast<cudaStream_t>(cuda_stream));
 }
 
 }  // extern "C"

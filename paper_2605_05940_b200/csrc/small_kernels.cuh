@@ -25,8 +25,81 @@ __device__ __forceinline__ int warp_sum_int(int v) {
   return v;
 }
 
+// Rounds-times-tiles cost of cutting `vtiles` vocabulary tiles into ns runs for `pairs` row
+// pairs on `clusters` CTA pairs; the smallest cost wins (ties: fewer runs).
+__host__ __device__ inline int choose_nsplit(int pairs, int vtiles, int clusters, int nsplit_max) {
+  int best = 1;
+  long long best_cost = -1;
+  for (int ns = 1; ns <= nsplit_max && ns <= vtiles; ++ns) {
+    const long long rounds = (static_cast<long long>(pairs) * ns + clusters - 1) / clusters;
+    const long long per = (vtiles + ns - 1) / ns;
+    const long long cost = rounds * per * 64 + ns;
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best = ns;
+    }
+  }
+  return best;
+}
+
+// One CTA.  Covers the tokens that carry loss (m_t = 1) with 128-row blocks: a block starts at
+// the first such token that no earlier block covers and spans the 128 packed rows from there,
+// so the blocks are disjoint and skip the masked stretches (prompts) between them.  Rows outside
+// every block have zero loss and zero gradient, and no tile of any later kernel is spent on
+// them.  list[i] = first row of block i; plan = {blocks, pairs of blocks, forward runs, 0}.
+// Tokens are first marked in a bitmap in shared memory (bitmap_words 32-bit words, enough for
+// T bits); when T is too large for that the blocks fall back to the aligned grid 0, 128, 256...
+// with the blocks that hold no loss token left out.
+__global__ void __launch_bounds__(1024) plan_blocks_kernel(int T, const uint8_t* __restrict__ mask,
+                                                           int bitmap_words, int vtiles, int nsplit_max,
+                                                           int clusters, int* plan, int* list) {
+  extern __shared__ uint32_t bitmap[];
+  const int words = (T + 31) / 32;
+  int nact = 0;
+  if (words <= bitmap_words) {
+    for (int w = threadIdx.x; w < words; w += blockDim.x) {
+      uint32_t bits = 0;
+      const int t0 = w * 32, t1 = min(T, t0 + 32);
+      if (mask == nullptr) {
+        bits = (t1 - t0 == 32) ? 0xffffffffu : ((1u << (t1 - t0)) - 1u);
+      } else {
+        for (int t = t0; t < t1; ++t) bits |= (mask[t] != 0 ? 1u : 0u) << (t - t0);
+      }
+      bitmap[w] = bits;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int t = 0;
+      while (t < T) {
+        // first loss token at or after t
+        int w = t >> 5;
+        uint32_t bits = bitmap[w] & (0xffffffffu << (t & 31));
+        while (bits == 0 && ++w < words) bits = bitmap[w];
+        if (bits == 0) break;
+        const int start = w * 32 + __ffs(bits) - 1;
+        list[nact++] = start;
+        t = start + 128;
+      }
+    }
+  } else if (threadIdx.x == 0) {
+    for (int b = 0; b * 128 < T; ++b) {
+      bool act = mask == nullptr;
+      for (int t = b * 128; t < min(T, b * 128 + 128) && !act; ++t) act = mask[t] != 0;
+      if (act) list[nact++] = b * 128;
+    }
+  }
+  if (threadIdx.x == 0) {
+    const int pairs = (nact + 1) / 2;
+    plan[0] = nact;
+    plan[1] = pairs;
+    plan[2] = choose_nsplit(pairs > 0 ? pairs : 1, vtiles, clusters, nsplit_max);
+    plan[3] = 0;
+  }
+}
+
 struct CombineParams {
-  int T, d, V, nslots;
+  int T, d, V;
+  const int* plan;        // plan[2] = forward runs; the partials hold 2 slots per run
   const float* partials;  // [nslots][kPFields][T]
   const __nv_bfloat16* hidden;
   const __nv_bfloat16* weight;
@@ -54,8 +127,23 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
   if (t >= p.T) return;
   const size_t fs = static_cast<size_t>(p.T);            // field stride
   const size_t ss = static_cast<size_t>(kPFields) * fs;  // slot stride
+  const int nslots = 2 * p.plan[2];
+  const bool on = p.loss_mask == nullptr || p.loss_mask[t] != 0;
+  if (!on) {
+    // no loss and no gradient here; the token's block may not even have been visited
+    if (lane == 0) {
+      p.kl[t] = 0.f;
+      if (p.nll_s != nullptr) p.nll_s[t] = 0.f;
+      if (p.nll_t != nullptr) p.nll_t[t] = 0.f;
+      // a huge log-sum-exp turns both probabilities of the gradient tile into exact zeros
+      p.lse2_a[t] = 1e30f;
+      p.lse2_b[t] = 1e30f;
+      p.coef[t] = 0.f;
+    }
+    return;
+  }
   float ma = -INFINITY, mb = -INFINITY;
-  for (int s = lane; s < p.nslots; s += 32) {
+  for (int s = lane; s < nslots; s += 32) {
     const float* q = p.partials + s * ss + t;
     ma = fmaxf(ma, q[kPMaxA * fs]);
     mb = fmaxf(mb, q[kPMaxB * fs]);
@@ -63,7 +151,7 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
   ma = warp_max(ma);
   mb = warp_max(mb);
   float sa = 0.f, cr = 0.f, sb = 0.f, sa1 = 0.f, sb1 = 0.f;
-  for (int s = lane; s < p.nslots; s += 32) {
+  for (int s = lane; s < nslots; s += 32) {
     const float* q = p.partials + s * ss + t;
     const float da = q[kPMaxA * fs] - ma, db = q[kPMaxB * fs] - mb;
     const float fa = exp2f(da), fb = exp2f(db);
@@ -83,7 +171,6 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
     sb1 = warp_sum(sb1);
   }
   const float lse_a = ma + log2f(sa), lse_b = mb + log2f(sb);
-  const bool on = p.loss_mask == nullptr || p.loss_mask[t] != 0;
 
   // label logits: O_S[t, y] = <H[t], W[y]> in fp32, O_T[t, y] read directly
   float nll_s = 0.f, nll_t = 0.f;
