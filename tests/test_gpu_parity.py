@@ -141,6 +141,26 @@ def test_all_tokens_masked_gives_zero_loss_and_zero_gradients():
     assert float(step.d_hidden.float().abs().max()) == 0 and float(step.d_weight.abs().max()) == 0
 
 
+@pytest.mark.parametrize("ranges", [
+    [(37, 90), (400, 401), (530, 790), (995, 1000)],     # six blocks, the last one runs past T
+    [(37, 90), (530, 790), (995, 1000)],                 # five: one CTA of the last pair has no block
+    [(0, 1)],                                            # a single loss token
+    [(999, 1000)],                                       # ... which is the very last row
+])
+def test_loss_tokens_in_scattered_stretches(ranges):
+    # the kernels only visit 128-row blocks that start at loss tokens; everything else must
+    # still come out as exact zeros, and nothing may leak between blocks
+    b = syn.scaled("c2", device=DEV, T=1000, d=128, V=1304, seed_base=11, min_len=50, max_len=400)
+    b.loss_mask[:] = 0
+    for lo, hi in ranges:
+        b.loss_mask[lo:hi] = 1
+    for dw in (torch.bfloat16, torch.float32):
+        step = run_step(b, dw_dtype=dw, grad_chunk_cols=512)
+        check_full_parity(b, step)
+    step = run_step(b)      # one chunk: dH stored directly
+    check_full_parity(b, step)
+
+
 def test_optional_inputs_may_be_null():
     b = _mini()
     H, W, Z, y, m = oracle_inputs(b)
