@@ -125,7 +125,17 @@ int npd_workspace_bytes(const npd_kd_args* args, size_t* out_bytes);
 int npd_phase_count(const npd_kd_args* args, int32_t* out_groups, int32_t* out_chunks);
 
 /* Fused forward + backward of the distillation term (see the struct).  `args`
- * is a HOST struct holding device pointers.  Enqueues on `cuda_stream`. */
+ * is a HOST struct holding device pointers.  Enqueues on `cuda_stream`.
+ *
+ * Tokens with loss_mask 0 have kl = nll = 0 and no gradient by definition; the kernels
+ * cover the tokens that carry loss with 128-row blocks (found on the device from
+ * loss_mask) and spend no work on the rest, so a batch with long masked prompts costs
+ * proportionally less.  Every output element is written all the same (zeros where
+ * nothing is computed).
+ *
+ * kl, nll_*, and d_weight are bitwise reproducible from run to run.  d_hidden is summed
+ * over vocabulary chunks with fp32 atomic adds whose order is not fixed: its last bits
+ * may differ between runs. */
 int npd_kd_fwd_bwd(const npd_kd_args* args, void* cuda_stream);
 
 /*
