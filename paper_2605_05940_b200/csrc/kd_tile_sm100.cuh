@@ -48,6 +48,9 @@ struct KdTileParams {
   const int* plan;  // {128-row blocks that hold loss tokens, pairs of them, forward runs, 0} (device)
   const int* list;  // first packed row of every such block, in order; a pair of CTAs owns two
                     // consecutive entries
+  int group_pairs;  // pairs of blocks per group: units are ordered group by group (within a group:
+                    // pair fastest, then run), so that the H rows the CTA pairs work on at
+                    // any one time stay in L2 while the W tiles are shared by a whole group
   int vt_begin;     // first 256-wide vocabulary tile of this launch
   int vt_count;     // number of vocabulary tiles of this launch; they are cut into runs (forward:
                     // plan[2] runs, gradient: one tile per run); a unit = (pair of blocks, run)
@@ -148,10 +151,13 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   // slot = this CTA's position in the block list, r = that block's first packed row, or -1
   // when the list has an odd length and this CTA has no block (it then stages the rows from 0
   // and writes nothing).
+  const int per_group = p.group_pairs * nsplit;  // units of a full group
   auto run_of = [&](int u, int& slot, int& r, int& s, int& vt0, int& vt1) {
-    slot = 2 * (u % pairs) + static_cast<int>(rank);
+    const int gi = u / per_group, local = u - gi * per_group;
+    const int gsize = min(p.group_pairs, pairs - gi * p.group_pairs);
+    s = local / gsize;
+    slot = 2 * (gi * p.group_pairs + local % gsize) + static_cast<int>(rank);
     r = slot < nact ? __ldg(p.list + slot) : -1;
-    s = u / pairs;
     vt0 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * s / nsplit);
     vt1 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * (s + 1) / nsplit);
   };

@@ -82,14 +82,16 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   pl->row_blocks = (a->T + 127) / 128;
   pl->vtiles = (a->V + 255) / 256;
   pl->clusters = std::max(sms / 2, 1);
-  // The fewer row pairs there are, the more runs are needed to fill the CTA pairs.
-  const int row_pairs = (pl->row_blocks + 1) / 2;
-  pl->nsplit_max = std::min(pl->vtiles, std::max(4, std::min(64, 8 * pl->clusters / row_pairs)));
+  // Up to 32 runs: enough to fill the CTA pairs evenly whatever the number of row pairs turns
+  // out to be; the partials cost 56 bytes per token and run.
+  pl->nsplit_max = std::min(pl->vtiles, 32);
   pl->grads = a->d_hidden != nullptr || a->d_weight != nullptr;
   // Vocabulary chunks of the backward: the bf16 logit-gradient block [T, chunk_cols] is the only
   // thing that travels between the gradient tiles and the two contractions.  Default: the
-  // largest chunk whose block stays within 256 MiB, chunks of (almost) equal width.
-  const long long budget = 256ll << 20;
+  // largest chunk whose block stays within 256 MiB or a sixteenth of the teacher logits' size,
+  // whichever is more (wide chunks keep the contraction units long and the number of passes
+  // over the dH accumulator small), chunks of (almost) equal width.
+  const long long budget = std::max<long long>(256ll << 20, static_cast<long long>(a->T) * a->V / 8);
   int max_tiles = a->grad_chunk_cols > 0
                       ? (a->grad_chunk_cols + 255) / 256
                       : static_cast<int>(std::max<long long>(8, budget / (512ll * a->T)));
@@ -99,10 +101,13 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   pl->chunk_cols = chunk_tiles * 256;
   pl->nchunks = (pl->vtiles + chunk_tiles - 1) / chunk_tiles;
   const int cc = pl->chunk_cols;
-  // dH = G W is cut along the chunk's columns into units of about 48 k-steps so that the
-  // pairs can be filled evenly; the partial products are added with fp32 atomics.
+  // dH = G W is cut along the chunk's columns (split-K, partial products added with fp32
+  // atomics) only as far as it takes to give every CTA pair about 8 units, and never into
+  // units shorter than 48 k-steps: short units pay the accumulator drain too often.
   const int ksteps_h = cc / 64;
-  pl->dh_ksplits = std::max(1, std::min(16, (ksteps_h + 24) / 48));
+  const long long tiles_h = static_cast<long long>((pl->row_blocks + 1) / 2) * ((a->d + 511) / 512);
+  const int want = static_cast<int>((8ll * pl->clusters + tiles_h - 1) / tiles_h);
+  pl->dh_ksplits = std::max(1, std::min(want, ksteps_h / 48));
   pl->dh_direct = pl->nchunks == 1 && pl->dh_ksplits == 1;
   size_t off = 0;
   pl->off_status = off;
@@ -331,6 +336,8 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   kp.ksteps = a->d / 64;
   kp.plan = plan;
   kp.list = list;
+  // a group's H rows (256 x d bf16 per pair) should fill at most a quarter of a 128 MB L2
+  kp.group_pairs = static_cast<int>(std::max<long long>(4, (32ll << 20) / (512ll * a->d)));
   kp.vt_begin = 0;
   kp.vt_count = pl.vtiles;
   kp.scale2 = scale2;
