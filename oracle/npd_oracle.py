@@ -29,6 +29,9 @@ cross-entropy L_theta of Eq. 3 is the token mean over the positions that carry
 loss; both ends of the keep interval are inclusive (Proximal Learning Zone,
 0 <= Delta <= threshold).
 
+The composite objective follows Eq. 1 with the cross-entropy at temperature 1; the
+top-k functions follow Eq. 2 as printed, with p_T the softmax of the k stored logits.
+
 Pins: every function below is pinned by tests/test_oracle_*.py against closed
 forms, finite differences, SciPy/PyTorch library routines, brute force and a
 hand-worked table (tests/golden/).  The one thing that cannot be pinned is the
@@ -49,6 +52,12 @@ __all__ = [
     "kd_backward",
     "kd_dhidden_rows",
     "kd_dweight_rows",
+    "composite_token_loss",
+    "composite_logit_gradient",
+    "composite_backward",
+    "topk_kd_token_losses",
+    "topk_kd_logit_gradient",
+    "topk_kd_backward",
     "validate_cu_seqlens",
     "segment_ids",
     "segment_stats",
@@ -177,6 +186,104 @@ def kd_dweight_rows(H, W, teacher_logits, loss_mask, tau, grad_scale, vocab_rows
         dO = kd_logit_gradient(Hg, W, Zg, np.asarray(loss_mask[t0:t1]), tau, grad_scale)
         out += np.matmul(dO[:, c].T, Hg)
     return out
+
+
+# --------------------------------------------------------------------------- #
+# Composite objective (Eq. 1): L_total = (1 - lambda) L_CE + lambda L_KD
+# --------------------------------------------------------------------------- #
+
+def composite_token_loss(kl, nll_s, lam: float):
+    """Eq. 1 token by token: (1 - lam) * CE_t + lam * KD_t, with CE_t the student's
+    negative log-likelihood of the label (temperature 1) and KD_t the distillation
+    term of Eq. 2, both already masked."""
+    return (1.0 - lam) * _f64(nll_s) + lam * _f64(kl)
+
+
+def composite_logit_gradient(H, W, teacher_logits, labels, loss_mask, tau: float,
+                             grad_scale: float, lam: float):
+    """dL/dO_S for L = grad_scale * sum_t m_t ((1 - lam) CE_t + lam KD_t)  (Eq. 1):
+
+        dO_S[t,c] = grad_scale * m_t * ( lam (p_S^tau(c) - p_T^tau(c)) / tau
+                                         + (1 - lam) [y_t>=0] (p_S^1(c) - [c = y_t]) )
+
+    p^tau = Softmax(./tau); the cross-entropy is taken at temperature 1."""
+    O_S = student_logits(H, W)
+    T, V = O_S.shape
+    labels = np.asarray(labels, dtype=np.int64)
+    m = np.asarray(loss_mask).astype(np.float64)[:, None]
+    d_kd = kd_logit_gradient(H, W, teacher_logits, loss_mask, tau, 1.0)
+    has = (labels >= 0).astype(np.float64)[:, None]
+    onehot = np.zeros((T, V))
+    onehot[np.arange(T)[labels >= 0], labels[labels >= 0]] = 1.0
+    d_ce = m * has * (np.exp(log_softmax(O_S)) - onehot)
+    return grad_scale * (lam * d_kd + (1.0 - lam) * d_ce)
+
+
+def composite_backward(H, W, teacher_logits, labels, loss_mask, tau: float, grad_scale: float,
+                       lam: float):
+    """dH = dO_S W, dW = dO_S^T H for the composite objective (Eq. 1, Algorithm 1 "Update")."""
+    dO = composite_logit_gradient(H, W, teacher_logits, labels, loss_mask, tau, grad_scale, lam)
+    return np.matmul(dO, _f64(W)), np.matmul(dO.T, _f64(H))
+
+
+# --------------------------------------------------------------------------- #
+# Eq. 2 as printed: the teacher is stored as its k largest logits per token
+# --------------------------------------------------------------------------- #
+
+def _topk_probs(topk_values, tau):
+    """p_T over the stored support: Softmax of the k stored logits / tau.  (Only the k
+    logits exist, so the teacher distribution is the one they define.)"""
+    return np.exp(log_softmax(_f64(topk_values) / tau))
+
+
+def topk_kd_token_losses(H, W, topk_values, topk_indices, labels, loss_mask, tau: float):
+    """Eq. 2 with the sum over V_top-k:
+
+        kl[t] = m_t * sum_{j<k} p_T(j) (log p_T(j) - log p_S(idx[t,j]))
+
+    p_T = Softmax over the k stored teacher logits (/tau), p_S = Softmax(O_S[t]/tau) over
+    the whole vocabulary, evaluated at the stored indices.  Also returns the student's
+    per-token cross-entropy at the labels (temperature 1), as kd_token_losses does.
+    Returns (kl, nll_s)."""
+    H = _f64(H)
+    T = H.shape[0]
+    O_S = student_logits(H, W)
+    idx = np.asarray(topk_indices, dtype=np.int64)
+    labels = np.asarray(labels, dtype=np.int64)
+    m = np.asarray(loss_mask).astype(bool)
+    p_T = _topk_probs(topk_values, tau)
+    logp_T = log_softmax(_f64(topk_values) / tau)
+    logp_S = np.take_along_axis(log_softmax(O_S / tau), idx, axis=1)
+    with np.errstate(invalid="ignore"):
+        terms = p_T * (logp_T - logp_S)
+    terms = np.where(p_T > 0.0, terms, 0.0)
+    kl = np.where(m, terms.sum(axis=1), 0.0)
+    has = m & (labels >= 0)
+    y = np.where(labels >= 0, labels, 0)
+    nll_s = np.where(has, -log_softmax(O_S)[np.arange(T), y], 0.0)
+    return kl, nll_s
+
+
+def topk_kd_logit_gradient(H, W, topk_values, topk_indices, loss_mask, tau: float,
+                           grad_scale: float):
+    """dL/dO_S for L = grad_scale * sum_t kl[t] of the top-k form:
+
+        dO_S[t,c] = grad_scale * m_t * (p_S(c) - sum_{j: idx[t,j]=c} p_T(j)) / tau
+
+    (the stored probabilities sum to one, so the student term keeps its full weight)."""
+    O_S = student_logits(H, W)
+    idx = np.asarray(topk_indices, dtype=np.int64)
+    p_S = np.exp(log_softmax(O_S / tau))
+    p_T = _topk_probs(topk_values, tau)
+    dense_T = np.zeros_like(p_S)
+    np.add.at(dense_T, (np.arange(O_S.shape[0])[:, None], idx), p_T)
+    m = np.asarray(loss_mask).astype(np.float64)[:, None]
+    return grad_scale * m * (p_S - dense_T) / tau
+
+
+def topk_kd_backward(H, W, topk_values, topk_indices, loss_mask, tau: float, grad_scale: float):
+    dO = topk_kd_logit_gradient(H, W, topk_values, topk_indices, loss_mask, tau, grad_scale)
+    return np.matmul(dO, _f64(W)), np.matmul(dO.T, _f64(H))
 
 
 # --------------------------------------------------------------------------- #

@@ -139,3 +139,124 @@ def test_row_restricted_gradients_match_the_full_ones():
     for grp in (0, 4, 5):
         got = orc.kd_dweight_rows(H, W, Zt, mask, 0.8, 0.1, vr, token_group=grp)
         assert np.allclose(got, dW[vr], rtol=1e-12, atol=1e-16)
+
+
+# ----------------------------------------------------------------------------------------------
+# Eq. 1: composite objective
+# ----------------------------------------------------------------------------------------------
+def _composite_loss(H, W, Zt, mask, y, tau, g, lam):
+    kl, ns, _ = orc.kd_token_losses(H, W, Zt, y, mask, tau)
+    return g * orc.composite_token_loss(kl, ns, lam).sum()
+
+
+@pytest.mark.parametrize("tau,g,lam", [(1.0, 1.0, 0.9), (2.5, 0.37, 0.5), (0.6, 1 / 3, 0.0), (1.7, 2.0, 1.0)])
+def test_composite_gradient_by_central_finite_differences(tau, g, lam):
+    H, W, Zt, mask, y = _problem(3)
+    y[2] = -100                                   # a loss token without a label: KD only
+    mask[2] = 1
+    dH, dW = orc.composite_backward(H, W, Zt, y, mask, tau, g, lam)
+    h = 1e-5
+    fdH = np.zeros_like(H)
+    for i in range(H.shape[0]):
+        for j in range(H.shape[1]):
+            Hp, Hm = H.copy(), H.copy()
+            Hp[i, j] += h
+            Hm[i, j] -= h
+            fdH[i, j] = (_composite_loss(Hp, W, Zt, mask, y, tau, g, lam) -
+                         _composite_loss(Hm, W, Zt, mask, y, tau, g, lam)) / (2 * h)
+    fdW = np.zeros_like(W)
+    for i in range(W.shape[0]):
+        for j in range(W.shape[1]):
+            Wp, Wm = W.copy(), W.copy()
+            Wp[i, j] += h
+            Wm[i, j] -= h
+            fdW[i, j] = (_composite_loss(H, Wp, Zt, mask, y, tau, g, lam) -
+                         _composite_loss(H, Wm, Zt, mask, y, tau, g, lam)) / (2 * h)
+    assert np.linalg.norm(fdH - dH) / np.linalg.norm(dH) < 1e-6
+    assert np.linalg.norm(fdW - dW) / np.linalg.norm(dW) < 1e-6
+
+
+def test_composite_reduces_to_its_two_terms():
+    H, W, Zt, mask, y = _problem(4)
+    tau, g = 1.3, 0.7
+    # lambda = 1: the distillation gradient alone
+    a = orc.composite_logit_gradient(H, W, Zt, y, mask, tau, g, 1.0)
+    assert np.allclose(a, orc.kd_logit_gradient(H, W, Zt, mask, tau, g), atol=1e-15)
+    # lambda = 0: torch's cross-entropy gradient on the masked tokens
+    Ht = torch.tensor(H, dtype=torch.float64, requires_grad=True)
+    Wt = torch.tensor(W, dtype=torch.float64, requires_grad=True)
+    logits = Ht @ Wt.T
+    ce = torch.nn.functional.cross_entropy(logits, torch.tensor(y), reduction="none")
+    (g * (ce * torch.tensor(mask, dtype=torch.float64)).sum()).backward()
+    dH, dW = orc.composite_backward(H, W, Zt, y, mask, tau, g, 0.0)
+    assert np.allclose(dH, Ht.grad.numpy(), atol=1e-12) and np.allclose(dW, Wt.grad.numpy(), atol=1e-12)
+    # linear in lambda, rows sum to zero, masked rows are zero
+    mid = orc.composite_logit_gradient(H, W, Zt, y, mask, tau, g, 0.25)
+    b = orc.composite_logit_gradient(H, W, Zt, y, mask, tau, g, 0.0)
+    assert np.allclose(mid, 0.25 * a + 0.75 * b, atol=1e-15)
+    assert np.abs(mid.sum(axis=1)).max() < 1e-12 and np.all(mid[mask == 0] == 0)
+
+
+# ----------------------------------------------------------------------------------------------
+# Eq. 2 as printed: top-k teacher support
+# ----------------------------------------------------------------------------------------------
+def _topk_problem(seed, T=6, d=5, V=11, k=4):
+    H, W, Zt, mask, y = _problem(seed, T=T, d=d, V=V)
+    idx = np.argsort(-Zt, axis=1)[:, :k]
+    vals = np.take_along_axis(Zt, idx, axis=1)
+    return H, W, Zt, mask, y, vals, idx
+
+
+@pytest.mark.parametrize("tau", [1.0, 2.0])
+def test_topk_form_equals_dense_form_with_minus_inf_outside_the_support(tau):
+    H, W, Zt, mask, y, vals, idx = _topk_problem(5)
+    dense = np.full_like(Zt, -np.inf)
+    np.put_along_axis(dense, idx, vals, axis=1)
+    kl_d, ns_d, _ = orc.kd_token_losses(H, W, dense, y, mask, tau)
+    kl_k, ns_k = orc.topk_kd_token_losses(H, W, vals, idx, y, mask, tau)
+    assert np.allclose(kl_k, kl_d, atol=1e-13) and np.allclose(ns_k, ns_d, atol=1e-15)
+    g_d = orc.kd_logit_gradient(H, W, dense, mask, tau, 0.4)
+    g_k = orc.topk_kd_logit_gradient(H, W, vals, idx, mask, tau, 0.4)
+    assert np.allclose(g_k, g_d, atol=1e-14)
+
+
+def test_topk_loss_brute_force_and_lower_bound():
+    H, W, Zt, mask, y, vals, idx = _topk_problem(6)
+    tau = 1.4
+    kl, _ = orc.topk_kd_token_losses(H, W, vals, idx, y, mask, tau)
+    O = H @ W.T
+    for t in range(H.shape[0]):
+        e = [np.exp(v / tau) for v in vals[t]]
+        pT = [x / sum(e) for x in e]
+        zs = [np.exp(o / tau) for o in O[t]]
+        pS = [z / sum(zs) for z in zs]
+        ref = sum(pT[j] * (np.log(pT[j]) - np.log(pS[idx[t, j]])) for j in range(len(pT)))
+        assert abs(kl[t] - (ref if mask[t] else 0.0)) < 1e-12
+        # the student's mass on the support is at most one: KL >= -log(that mass) >= 0
+        mass = sum(pS[c] for c in idx[t])
+        if mask[t]:
+            assert kl[t] >= -np.log(mass) - 1e-12 >= -1e-12
+
+
+def test_topk_gradient_by_central_finite_differences():
+    H, W, Zt, mask, y, vals, idx = _topk_problem(7)
+    tau, g = 1.8, 0.6
+    dH, dW = orc.topk_kd_backward(H, W, vals, idx, mask, tau, g)
+    loss = lambda H_, W_: g * orc.topk_kd_token_losses(H_, W_, vals, idx, y, mask, tau)[0].sum()
+    h = 1e-5
+    fdH = np.zeros_like(H)
+    for i in range(H.shape[0]):
+        for j in range(H.shape[1]):
+            Hp, Hm = H.copy(), H.copy()
+            Hp[i, j] += h
+            Hm[i, j] -= h
+            fdH[i, j] = (loss(Hp, W) - loss(Hm, W)) / (2 * h)
+    fdW = np.zeros_like(W)
+    for i in range(W.shape[0]):
+        for j in range(W.shape[1]):
+            Wp, Wm = W.copy(), W.copy()
+            Wp[i, j] += h
+            Wm[i, j] -= h
+            fdW[i, j] = (loss(H, Wp) - loss(H, Wm)) / (2 * h)
+    assert np.linalg.norm(fdH - dH) / np.linalg.norm(dH) < 1e-6
+    assert np.linalg.norm(fdW - dW) / np.linalg.norm(dW) < 1e-6
