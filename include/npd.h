@@ -62,7 +62,15 @@ enum { NPD_DTYPE_BF16 = 0, NPD_DTYPE_F32 = 1 };
 
 /* flags of npd_kd_args */
 enum {
-  NPD_KD_ACCUMULATE_DW = 1  /* add into d_weight instead of overwriting it (f32 d_weight only) */
+  NPD_KD_ACCUMULATE_DW = 1, /* add into d_weight instead of overwriting it (f32 d_weight only) */
+  NPD_KD_COMPOSITE_LOSS = 2 /* gradients of the composite objective of Eq. 1,
+                               L_total = (1 - lambda) L_CE + lambda L_KD with lambda = kd_lambda:
+                                 dO_S[t,c] = grad_scale * m_t * ( lambda (p_S - p_T) / tau
+                                             + (1 - lambda) [y_t>=0] (Softmax(O_S[t])[c] - [c = y_t]) )
+                               (cross-entropy at temperature 1).  Needs labels.  The per-token
+                               outputs are unchanged: the loss value of a token is
+                               (1 - lambda) * nll_student[t] + lambda * kl[t].  Without the flag
+                               the gradients are those of Eq. 2 alone (lambda = 1). */
 };
 
 /*
@@ -101,7 +109,8 @@ typedef struct npd_kd_args {
   int32_t grad_chunk_cols;   /* vocabulary columns of logit-gradient tiles that may be in
                                 flight between the gradient kernel and the two
                                 contractions; 0 = library default.  Bounds the scratch. */
-  int32_t reserved1;
+  float kd_lambda;           /* lambda of Eq. 1 in [0,1]; read only with NPD_KD_COMPOSITE_LOSS
+                                (the paper trains with 0.9) */
   void* workspace;           /* >= npd_workspace_bytes(), 1024-byte aligned         */
   size_t workspace_bytes;
   /* Optional timing hooks.  HOST array of n_phase_events cudaEvent_t (as void*), or NULL.

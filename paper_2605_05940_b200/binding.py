@@ -21,6 +21,7 @@ NPD_EINVAL, NPD_ESHAPE, NPD_EALIGN, NPD_ESEQ, NPD_EARCH = -1, -2, -3, -4, -5
 NPD_EWORKSPACE, NPD_ECUDA, NPD_ETIMEOUT, NPD_EUNSUPPORTED = -6, -7, -8, -9
 NPD_DTYPE_BF16, NPD_DTYPE_F32 = 0, 1
 NPD_KD_ACCUMULATE_DW = 1
+NPD_KD_COMPOSITE_LOSS = 2
 NPD_SELECT_TEACHER_IFD_LE_1 = 1
 NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32 = range(4)
 
@@ -48,7 +49,7 @@ class npd_kd_args(C.Structure):
         ("kl", C.c_void_p), ("nll_student", C.c_void_p), ("nll_teacher", C.c_void_p),
         ("d_hidden", C.c_void_p), ("d_weight", C.c_void_p),
         ("d_weight_dtype", C.c_int32), ("flags", C.c_int32),
-        ("grad_chunk_cols", C.c_int32), ("reserved1", C.c_int32),
+        ("grad_chunk_cols", C.c_int32), ("kd_lambda", C.c_float),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("phase_events", C.POINTER(C.c_void_p)), ("n_phase_events", C.c_int32), ("reserved2", C.c_int32),
     ]
@@ -106,7 +107,7 @@ def _check(rc: int, where: str):
 
 def make_kd_args(hidden, weight, teacher, *, cu_seqlens=None, loss_mask=None, labels=None,
                  temperature=1.0, grad_scale=1.0, kl=None, nll_student=None, nll_teacher=None,
-                 d_hidden=None, d_weight=None, flags=0, grad_chunk_cols=0,
+                 d_hidden=None, d_weight=None, flags=0, grad_chunk_cols=0, kd_lambda=None,
                  workspace=None) -> npd_kd_args:
     """Fill an npd_kd_args from tensors (device tensors, or host tensors for the
     `host` argument of npd_kd_fwd_bwd_host)."""
@@ -125,6 +126,9 @@ def make_kd_args(hidden, weight, teacher, *, cu_seqlens=None, loss_mask=None, la
     a.d_weight_dtype = (NPD_DTYPE_F32 if d_weight is not None and d_weight.dtype == torch.float32
                         else NPD_DTYPE_BF16)
     a.flags, a.grad_chunk_cols = int(flags), int(grad_chunk_cols)
+    if kd_lambda is not None:       # composite objective of Eq. 1
+        a.flags |= NPD_KD_COMPOSITE_LOSS
+        a.kd_lambda = float(kd_lambda)
     if workspace is not None:
         a.workspace, a.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     return a
@@ -223,7 +227,8 @@ class KDStep:
     """Holds the output and workspace tensors of one problem shape and runs the
     fused step on them; a convenience over the raw calls."""
 
-    def __init__(self, batch, *, grads=True, dw_dtype=torch.bfloat16, grad_chunk_cols=0, grad_scale=None):
+    def __init__(self, batch, *, grads=True, dw_dtype=torch.bfloat16, grad_chunk_cols=0, grad_scale=None,
+                 kd_lambda=None):
         dev = batch.hidden.device
         T, d, V = batch.T, batch.d, batch.V
         f32 = dict(dtype=torch.float32, device=dev)
@@ -240,7 +245,8 @@ class KDStep:
         self._kw = dict(cu_seqlens=batch.cu_seqlens, loss_mask=batch.loss_mask, labels=batch.labels,
                         temperature=batch.tau, grad_scale=self.grad_scale, kl=self.kl,
                         nll_student=self.nll_student, nll_teacher=self.nll_teacher,
-                        d_hidden=self.d_hidden, d_weight=self.d_weight, grad_chunk_cols=grad_chunk_cols)
+                        d_hidden=self.d_hidden, d_weight=self.d_weight, grad_chunk_cols=grad_chunk_cols,
+                        kd_lambda=kd_lambda)
         probe = make_kd_args(batch.hidden, batch.weight, batch.teacher, **self._kw)
         nbytes = npd_workspace_bytes(probe)
         self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)

@@ -11,9 +11,11 @@
 //              as running (max, sum, sum*(difference)) per token and written as
 //              partial results per vocabulary split.
 //   kGradient: with the per-token log-sum-exps known, the logit gradient
-//              dO_S = coef_t (p_S - p_T), coef_t = grad_scale*m_t/tau (gradient of
+//              dO_S = coef_t (p_S - p_T), coef_t = grad_scale*m_t*lambda/tau (gradient of
 //              Eq. 2), rounded to bf16 and stored to a scratch block that the two
-//              backward contractions read.
+//              backward contractions read.  With kComposite the cross-entropy term of
+//              Eq. 1 is added: + cce_t (Softmax(O_S)[c] - [c = y_t]),
+//              cce_t = grad_scale*m_t*(1-lambda).
 //
 // Two CTAs on neighbouring SMs (a cluster of 2) work as a pair on a 256-token x 256-column
 // tile with tcgen05 .cta_group::2: each CTA stages its own 128 token rows of H and its own
@@ -61,7 +63,11 @@ struct KdTileParams {
   // gradient
   const float* lse2_a;  // [T] log2-sum-exp2 of the scaled teacher logits
   const float* lse2_b;  // [T] same for the student
-  const float* coef;    // [T] grad_scale * m_t / tau
+  const float* coef;    // [T] grad_scale * m_t * lambda / tau
+  // composite objective only (Eq. 1)
+  const float* coef_ce;   // [T] grad_scale * m_t * [y_t >= 0] * (1 - lambda)
+  const float* lse2_b1;   // [T] log2-sum-exp2 of the student logits * log2(e) (temperature 1)
+  const int32_t* labels;  // [T]
   int g_col0;           // vocabulary column that scratch column 0 holds; scratch row = position in
                         // the block list * 128 + row within the block
   int* status;
@@ -91,7 +97,7 @@ constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;
 constexpr float kNegClamp = -30000.0f;
 }  // namespace kd_cfg
 
-template <int kMode, bool kTauIsOne>
+template <int kMode, bool kTauIsOne, bool kComposite>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kd_cfg::THREADS, 1)
 kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                const __grid_constant__ CUtensorMap tmap_t, const __grid_constant__ CUtensorMap tmap_g,
@@ -272,10 +278,17 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       float m_a = -INFINITY, s_a = 0.f, cross = 0.f, m_b = -INFINITY, s_b = 0.f, s_a1 = 0.f, s_b1 = 0.f;
       // rows without a token (beyond T, or a CTA without a block): probabilities 0, gradient 0
       float g_lse_a = 1e30f, g_lse_b = 1e30f, g_coef = 0.f;
+      float g_cce = 0.f, g_lse_b1 = 1e30f;  // cross-entropy term of the composite objective
+      int g_y = -1;
       if (kMode == kGradient && row < p.T) {
         g_lse_a = p.lse2_a[row];
         g_lse_b = p.lse2_b[row];
         g_coef = p.coef[row];
+        if (kComposite) {
+          g_cce = p.coef_ce[row];
+          g_lse_b1 = p.lse2_b1[row];
+          g_y = g_cce != 0.f ? p.labels[row] : -1;
+        }
       }
       for (int vt = vt0; vt < vt1 && ok; ++vt, ++tile) {
         const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
@@ -356,12 +369,20 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             } else {
               // gradient tile: dO_S = coef * (p_S - p_T), written back in place over the teacher
               uint32_t packed[16];
+              const int yi = kComposite ? g_y - col0 : -1;  // label's place in this chunk, if any
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
-                float g0 = g_coef * (ex2f(fmaf(__uint_as_float(acc[i]), p.scale2, -g_lse_b)) -
-                                     ex2f(fmaf(zt[i], p.scale2, -g_lse_a)));
-                float g1 = g_coef * (ex2f(fmaf(__uint_as_float(acc[i + 1]), p.scale2, -g_lse_b)) -
-                                     ex2f(fmaf(zt[i + 1], p.scale2, -g_lse_a)));
+                const float s0 = __uint_as_float(acc[i]), s1 = __uint_as_float(acc[i + 1]);
+                const float ps0 = ex2f(fmaf(s0, p.scale2, -g_lse_b)), ps1 = ex2f(fmaf(s1, p.scale2, -g_lse_b));
+                float g0 = g_coef * (ps0 - ex2f(fmaf(zt[i], p.scale2, -g_lse_a)));
+                float g1 = g_coef * (ps1 - ex2f(fmaf(zt[i + 1], p.scale2, -g_lse_a)));
+                if (kComposite) {
+                  // at temperature 1 the two student softmaxes are the same
+                  const float q0 = kTauIsOne ? ps0 : ex2f(fmaf(s0, 1.4426950408889634f, -g_lse_b1));
+                  const float q1 = kTauIsOne ? ps1 : ex2f(fmaf(s1, 1.4426950408889634f, -g_lse_b1));
+                  g0 = fmaf(g_cce, q0 - (i == yi ? 1.f : 0.f), g0);
+                  g1 = fmaf(g_cce, q1 - (i + 1 == yi ? 1.f : 0.f), g1);
+                }
                 if (i >= nvalid) g0 = 0.f;
                 if (i + 1 >= nvalid) g1 = 0.f;
                 packed[i >> 1] = pack_bf16x2(g0, g1);

@@ -75,7 +75,8 @@ struct Plan {
   int dh_ksplits;     // split-K of the dH product of a full chunk
   bool dh_direct;     // dH stored straight to the output (one chunk, no split-K); else fp32 atomics
   bool grads;
-  size_t off_status, off_plan, off_list, off_partials, off_lse_a, off_lse_b, off_coef, off_g, off_dh, total;
+  size_t off_status, off_plan, off_list, off_partials, off_lse_a, off_lse_b, off_coef, off_coef_ce,
+      off_lse_b1, off_g, off_dh, total;
 };
 
 int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
@@ -124,6 +125,13 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   off = align_up(off + sizeof(float) * a->T, 1024);
   pl->off_coef = off;
   off = align_up(off + sizeof(float) * a->T, 1024);
+  pl->off_coef_ce = pl->off_lse_b1 = off;
+  if (a->flags & NPD_KD_COMPOSITE_LOSS) {
+    pl->off_coef_ce = off;
+    off = align_up(off + sizeof(float) * a->T, 1024);
+    pl->off_lse_b1 = off;
+    off = align_up(off + sizeof(float) * a->T, 1024);
+  }
   pl->off_g = off;
   pl->off_dh = off;
   if (pl->grads) {
@@ -149,6 +157,10 @@ int check_args(const npd_kd_args* a, bool need_pointers) {
   if ((a->ldh % 8) || (a->ldw % 8) || (a->ldt % 8)) return NPD_EALIGN;
   if ((a->d_hidden == nullptr) != (a->d_weight == nullptr)) return NPD_EINVAL;
   if ((a->flags & NPD_KD_ACCUMULATE_DW) && a->d_weight_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
+  if (a->flags & NPD_KD_COMPOSITE_LOSS) {
+    if (!(a->kd_lambda >= 0.f && a->kd_lambda <= 1.f)) return NPD_EINVAL;
+    if (need_pointers && a->labels == nullptr) return NPD_EINVAL;
+  }
   if (!need_pointers) return NPD_OK;
   if (a->hidden == nullptr || a->weight == nullptr || a->teacher == nullptr || a->kl == nullptr)
     return NPD_EINVAL;
@@ -228,10 +240,12 @@ int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const
 }
 
 template <int kMode>
-int launch_kd_tile(bool tau_one, const CUtensorMap& mh, const CUtensorMap& mw, const CUtensorMap& mt,
+int launch_kd_tile(bool tau_one, bool composite, const CUtensorMap& mh, const CUtensorMap& mw, const CUtensorMap& mt,
                    const CUtensorMap& mg, const KdTileParams& kp, int sms, cudaStream_t st) {
   using namespace kd_cfg;
-  auto k = tau_one ? kd_tile_kernel<kMode, true> : kd_tile_kernel<kMode, false>;
+  auto k = tau_one ? kd_tile_kernel<kMode, true, false> : kd_tile_kernel<kMode, false, false>;
+  if (kMode == kGradient && composite)
+    k = tau_one ? kd_tile_kernel<kMode, true, true> : kd_tile_kernel<kMode, false, true>;
   if (set_smem(k, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
   // the number of units is only known on the device: always one CTA pair per two SMs
   const int grid = 2 * std::max(sms / 2, 1);
@@ -295,6 +309,9 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   float* lse_a = reinterpret_cast<float*>(ws + pl.off_lse_a);
   float* lse_b = reinterpret_cast<float*>(ws + pl.off_lse_b);
   float* coef = reinterpret_cast<float*>(ws + pl.off_coef);
+  const bool composite = (a->flags & NPD_KD_COMPOSITE_LOSS) != 0;
+  float* coef_ce = composite ? reinterpret_cast<float*>(ws + pl.off_coef_ce) : nullptr;
+  float* lse_b1 = composite ? reinterpret_cast<float*>(ws + pl.off_lse_b1) : nullptr;
   if (cudaMemsetAsync(status, 0, 64, st) != cudaSuccess) return NPD_ECUDA;
   PhaseRecorder rec{a->phase_events, a->n_phase_events, 0, st};
 
@@ -344,7 +361,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   kp.tau = a->temperature;
   kp.partials = partials;
   kp.status = status;
-  if ((rc = launch_kd_tile<kForward>(tau_one, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
+  if ((rc = launch_kd_tile<kForward>(tau_one, false, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
   rec.mark();
 
   CombineParams cp{};
@@ -370,6 +387,9 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   cp.lse2_a = lse_a;
   cp.lse2_b = lse_b;
   cp.coef = coef;
+  cp.lambda = composite ? a->kd_lambda : 1.f;
+  cp.coef_ce = coef_ce;
+  cp.lse2_b1 = lse_b1;
   if (tau_one)
     kd_combine_kernel<true><<<(a->T + 7) / 8, 256, 0, st>>>(cp);
   else
@@ -407,8 +427,11 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     gp.lse2_a = lse_a;
     gp.lse2_b = lse_b;
     gp.coef = coef;
+    gp.coef_ce = coef_ce;
+    gp.lse2_b1 = lse_b1;
+    gp.labels = a->labels;
     gp.g_col0 = col0;
-    if ((rc = launch_kd_tile<kGradient>(tau_one, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
+    if ((rc = launch_kd_tile<kGradient>(tau_one, composite, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
     rec.mark();
 
     GemmProblem pr[2] = {};

@@ -114,6 +114,11 @@ struct CombineParams {
   float* lse2_a;
   float* lse2_b;
   float* coef;
+  // composite objective (Eq. 1): lambda weighs the distillation term, 1 - lambda the
+  // cross-entropy; coef_ce / lse2_b1 are NULL when the objective is Eq. 2 alone (lambda = 1)
+  float lambda;
+  float* coef_ce;
+  float* lse2_b1;
 };
 
 // One warp per token.  Merges the per-split online-softmax partials into the token's
@@ -139,6 +144,10 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
       p.lse2_a[t] = 1e30f;
       p.lse2_b[t] = 1e30f;
       p.coef[t] = 0.f;
+      if (p.coef_ce != nullptr) {
+        p.coef_ce[t] = 0.f;
+        p.lse2_b1[t] = 1e30f;
+      }
     }
     return;
   }
@@ -174,9 +183,11 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
 
   // label logits: O_S[t, y] = <H[t], W[y]> in fp32, O_T[t, y] read directly
   float nll_s = 0.f, nll_t = 0.f;
+  bool has_label = false;
   if (p.labels != nullptr) {
     const int y = p.labels[t];
     if (on && y >= 0 && y < p.V) {
+      has_label = true;
       const uint4* h4 = reinterpret_cast<const uint4*>(p.hidden + static_cast<size_t>(t) * p.ldh);
       const uint4* w4 = reinterpret_cast<const uint4*>(p.weight + static_cast<size_t>(y) * p.ldw);
       float dot = 0.f;
@@ -207,7 +218,11 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
     if (p.nll_t != nullptr) p.nll_t[t] = nll_t;
     p.lse2_a[t] = lse_a;
     p.lse2_b[t] = lse_b;
-    p.coef[t] = on ? p.grad_scale / p.tau : 0.f;
+    p.coef[t] = on ? p.grad_scale * p.lambda / p.tau : 0.f;
+    if (p.coef_ce != nullptr) {
+      p.coef_ce[t] = has_label ? p.grad_scale * (1.f - p.lambda) : 0.f;
+      p.lse2_b1[t] = kTauIsOne ? lse_b : mb * p.tau + log2f(sb1);
+    }
   }
 }
 

@@ -105,6 +105,25 @@ def test_config4_short_segments_full_segment_count_and_selection():
     assert 0.2 < frac < 0.9       # the 80th-percentile threshold keeps a real subset
 
 
+@pytest.mark.parametrize("tau,lam", [(1.0, 0.9), (2.0, 0.5), (1.0, 0.0), (1.5, 1.0)])
+def test_composite_objective_gradients(tau, lam):
+    # Eq. 1: (1 - lambda) CE + lambda KD; the per-token outputs do not change
+    b = syn.scaled("c2", device=DEV, T=700, d=128, V=3000, min_len=20, max_len=300)
+    b.tau = tau
+    step = run_step(b, kd_lambda=lam, dw_dtype=torch.float32, grad_chunk_cols=1024)
+    H, W, Z, y, m = oracle_inputs(b)
+    kl, ns, nt = orc.kd_token_losses(H, W, Z, y, m, tau)
+    assert_losses_close(host(step.kl), kl, "kl")
+    assert_losses_close(host(step.nll_student), ns, "nll_student")
+    dH, dW = orc.composite_backward(H, W, Z, y, m, tau, step.grad_scale, lam)
+    assert frob(host(step.d_hidden), dH) <= GRAD_FROB
+    assert frob(host(step.d_weight), dW) <= GRAD_FROB
+    assert np.all(host(step.d_hidden)[m == 0] == 0)
+    if lam == 1.0:      # the flag with lambda = 1 is the plain distillation gradient
+        plain = run_step(b, dw_dtype=torch.float32, grad_chunk_cols=1024)
+        assert torch.equal(plain.d_weight, step.d_weight)
+
+
 def test_runs_are_bitwise_reproducible():
     b = syn.scaled("c2", device=DEV, T=700, d=128, V=3000, min_len=20, max_len=300)
     s1 = run_step(b, grad_chunk_cols=1024)
