@@ -87,7 +87,8 @@ typedef struct npd_kd_args {
   int32_t T, d, V, S;
   const void* hidden;        /* bf16 [T, ldh]   H                                  */
   const void* weight;        /* bf16 [V, ldw]   W (LM head, no bias)               */
-  const void* teacher;       /* bf16 [T, ldt]   O_T, ldt >= V; columns >= V ignored */
+  const void* teacher;       /* bf16 [T, ldt]   O_T, ldt >= V; columns >= V ignored
+                                (not read when topk > 0, see the end of the struct) */
   int64_t ldh, ldw, ldt;
   int32_t teacher_dtype;     /* NPD_DTYPE_BF16 (NPD_DTYPE_F32: NPD_EUNSUPPORTED)    */
   int32_t reserved0;
@@ -122,6 +123,18 @@ typedef struct npd_kd_args {
   void* const* phase_events;
   int32_t n_phase_events;
   int32_t reserved2;
+  /* Teacher stored as its largest logits per token (Eq. 2 as printed: the sum runs over
+     V_top-k).  With topk > 0 the dense `teacher` is not read (may be NULL) and
+       p_T      = Softmax(topk_values[t, :] / tau) over the topk stored logits,
+       kl[t]    = m_t * sum_j p_T(j) (log p_T(j) - log p_S(topk_indices[t,j])),
+       dO_S[t,c] = grad_scale * m_t * lambda * (p_S(c) - sum_{j: idx[t,j]=c} p_T(j)) / tau,
+     p_S still the softmax over the whole vocabulary.  nll_teacher must be NULL (the stored
+     logits do not define the teacher's probability of an arbitrary label).  A stored logit
+     of -inf marks an unused entry.  topk <= 16; indices must lie in [0, V). */
+  const float* topk_values;    /* f32 [T, topk] */
+  const int32_t* topk_indices; /* [T, topk]     */
+  int32_t topk;                /* 0 = dense teacher */
+  int32_t reserved3;
 } npd_kd_args;
 
 /* HOST.  Bytes of workspace npd_kd_fwd_bwd needs for these arguments (pointers

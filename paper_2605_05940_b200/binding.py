@@ -52,6 +52,7 @@ class npd_kd_args(C.Structure):
         ("grad_chunk_cols", C.c_int32), ("kd_lambda", C.c_float),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("phase_events", C.POINTER(C.c_void_p)), ("n_phase_events", C.c_int32), ("reserved2", C.c_int32),
+        ("topk_values", C.c_void_p), ("topk_indices", C.c_void_p), ("topk", C.c_int32), ("reserved3", C.c_int32),
     ]
 
 
@@ -108,7 +109,7 @@ def _check(rc: int, where: str):
 def make_kd_args(hidden, weight, teacher, *, cu_seqlens=None, loss_mask=None, labels=None,
                  temperature=1.0, grad_scale=1.0, kl=None, nll_student=None, nll_teacher=None,
                  d_hidden=None, d_weight=None, flags=0, grad_chunk_cols=0, kd_lambda=None,
-                 workspace=None) -> npd_kd_args:
+                 topk_values=None, topk_indices=None, workspace=None) -> npd_kd_args:
     """Fill an npd_kd_args from tensors (device tensors, or host tensors for the
     `host` argument of npd_kd_fwd_bwd_host)."""
     a = npd_kd_args()
@@ -117,8 +118,15 @@ def make_kd_args(hidden, weight, teacher, *, cu_seqlens=None, loss_mask=None, la
     a.V = weight.shape[0]
     a.S = 0 if cu_seqlens is None else cu_seqlens.numel() - 1
     a.hidden, a.weight, a.teacher = _ptr(hidden), _ptr(weight), _ptr(teacher)
-    a.ldh, a.ldw, a.ldt = hidden.stride(0), weight.stride(0), teacher.stride(0)
-    a.teacher_dtype = NPD_DTYPE_F32 if teacher.dtype == torch.float32 else NPD_DTYPE_BF16
+    a.ldh, a.ldw = hidden.stride(0), weight.stride(0)
+    if teacher is not None:
+        a.ldt = teacher.stride(0)
+        a.teacher_dtype = NPD_DTYPE_F32 if teacher.dtype == torch.float32 else NPD_DTYPE_BF16
+    else:                           # top-k teacher: f32 [T,k] logits and int32 [T,k] indices
+        a.ldt = (a.V + 7) // 8 * 8
+        a.teacher_dtype = NPD_DTYPE_BF16
+    if topk_values is not None:
+        a.topk_values, a.topk_indices, a.topk = _ptr(topk_values), _ptr(topk_indices), topk_values.shape[1]
     a.cu_seqlens, a.loss_mask, a.labels = _ptr(cu_seqlens), _ptr(loss_mask), _ptr(labels)
     a.temperature, a.grad_scale = float(temperature), float(grad_scale)
     a.kl, a.nll_student, a.nll_teacher = _ptr(kl), _ptr(nll_student), _ptr(nll_teacher)
@@ -228,14 +236,15 @@ class KDStep:
     fused step on them; a convenience over the raw calls."""
 
     def __init__(self, batch, *, grads=True, dw_dtype=torch.bfloat16, grad_chunk_cols=0, grad_scale=None,
-                 kd_lambda=None):
+                 kd_lambda=None, topk_values=None, topk_indices=None):
         dev = batch.hidden.device
         T, d, V = batch.T, batch.d, batch.V
         f32 = dict(dtype=torch.float32, device=dev)
         self.batch = batch
         self.kl = torch.empty(T, **f32)
         self.nll_student = torch.empty(T, **f32)
-        self.nll_teacher = torch.empty(T, **f32)
+        self.nll_teacher = torch.empty(T, **f32) if topk_values is None else None
+        self.topk_values, self.topk_indices = topk_values, topk_indices
         # the gradients use the row strides of the tensors they belong to (ldh, ldw)
         self.d_hidden = (torch.empty_strided((T, d), (batch.hidden.stride(0), 1), dtype=torch.bfloat16,
                                              device=dev) if grads else None)
@@ -246,13 +255,14 @@ class KDStep:
                         temperature=batch.tau, grad_scale=self.grad_scale, kl=self.kl,
                         nll_student=self.nll_student, nll_teacher=self.nll_teacher,
                         d_hidden=self.d_hidden, d_weight=self.d_weight, grad_chunk_cols=grad_chunk_cols,
-                        kd_lambda=kd_lambda)
-        probe = make_kd_args(batch.hidden, batch.weight, batch.teacher, **self._kw)
+                        kd_lambda=kd_lambda, topk_values=topk_values, topk_indices=topk_indices)
+        teacher = batch.teacher if topk_values is None else None
+        probe = make_kd_args(batch.hidden, batch.weight, teacher, **self._kw)
         nbytes = npd_workspace_bytes(probe)
         self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device=dev)
         off = (-self.workspace.data_ptr()) % 1024
         self._ws_view = self.workspace[off: off + nbytes]
-        self.args = make_kd_args(batch.hidden, batch.weight, batch.teacher, workspace=self._ws_view,
+        self.args = make_kd_args(batch.hidden, batch.weight, teacher, workspace=self._ws_view,
                                  **self._kw)
 
     def run(self, stream=None):

@@ -33,6 +33,11 @@
 //   warps 4-11  epilogue; warp w reads TMEM lanes 32*(w%4).., columns 128*((w-4)/4)..
 //               so every thread owns one token row and half of the tile's columns.
 // All exponentials are taken in base 2 on logits pre-scaled by log2(e)/tau.
+//
+// kSparse: the teacher is given as its k largest logits per token (Eq. 2 as printed) instead
+// of a dense row.  The forward then keeps the student's statistics only (the k teacher terms
+// are evaluated per token afterwards), warp 2 has nothing to stream, and the gradient tile is
+// coef_t p_S minus the k stored teacher probabilities at their columns.
 #pragma once
 
 #include "ptx_sm100.cuh"
@@ -68,6 +73,10 @@ struct KdTileParams {
   const float* coef_ce;   // [T] grad_scale * m_t * [y_t >= 0] * (1 - lambda)
   const float* lse2_b1;   // [T] log2-sum-exp2 of the student logits * log2(e) (temperature 1)
   const int32_t* labels;  // [T]
+  // top-k teacher only (kSparse)
+  const int32_t* tk_idx;  // [T, topk] vocabulary indices of the stored teacher logits
+  const float* tk_cp;     // [T, topk] coef_t * p_T(j): what the gradient subtracts at column idx[t,j]
+  int topk;               // <= kMaxTopK
   int g_col0;           // vocabulary column that scratch column 0 holds; scratch row = position in
                         // the block list * 128 + row within the block
   int* status;
@@ -95,9 +104,10 @@ constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;
 // any sane row, and small enough in magnitude that fp32 still resolves differences of scaled
 // logits near it (a huge stand-in would turn "x*scale - max" into a rounding-error blow-up).
 constexpr float kNegClamp = -30000.0f;
+constexpr int kMaxTopK = 16;  // stored teacher logits per token the sparse path keeps in registers
 }  // namespace kd_cfg
 
-template <int kMode, bool kTauIsOne, bool kComposite>
+template <int kMode, bool kTauIsOne, bool kComposite, bool kSparse>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kd_cfg::THREADS, 1)
 kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                const __grid_constant__ CUtensorMap tmap_t, const __grid_constant__ CUtensorMap tmap_g,
@@ -233,7 +243,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     }
   } else if (warp == 2) {
     // ---------------------- teacher producer ----------------------
-    if (lane == 0) {
+    if (!kSparse && lane == 0) {
       uint32_t zit = 0;  // sub-tile pairs issued; both halves advance together
       bool ok = true;
       for (int u = cluster_id; u < units && ok; u += num_clusters) {
@@ -290,6 +300,17 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           g_y = g_cce != 0.f ? p.labels[row] : -1;
         }
       }
+      // top-k teacher: this row's stored columns and what to subtract there
+      int tki[kMaxTopK];
+      float tkc[kMaxTopK];
+      if (kSparse && kMode == kGradient) {
+#pragma unroll
+        for (int j = 0; j < kMaxTopK; ++j) {
+          const bool have = row < p.T && j < p.topk;
+          tki[j] = have ? p.tk_idx[static_cast<size_t>(row) * p.topk + j] : -1;
+          tkc[j] = have ? p.tk_cp[static_cast<size_t>(row) * p.topk + j] : 0.f;
+        }
+      }
       for (int vt = vt0; vt < vt1 && ok; ++vt, ++tile) {
         const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * buf, tph, abort_flag));
@@ -300,8 +321,10 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         for (int j = 0; j < BN / 2 / ZSUB_COLS && ok; ++j, ++zit) {
           const uint32_t q = zit % ZQ, zph = (zit / ZQ) & 1;
           const uint32_t bi = 8 * (half * ZQ + q);
-          ok = __all_sync(0xffffffffu, mbar_wait(zfull0 + bi, zph, abort_flag));
-          if (!ok) break;
+          if (!kSparse) {
+            ok = __all_sync(0xffffffffu, mbar_wait(zfull0 + bi, zph, abort_flag));
+            if (!ok) break;
+          }
           uint8_t* zrow = smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES + row_local * 128;
           const int sub_col0 = vt * BN + half * (BN / 2) + j * ZSUB_COLS;
 #pragma unroll 1
@@ -310,22 +333,48 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             uint32_t acc[32];
             tmem_ld32(taddr + j * ZSUB_COLS + c * 32, acc);
             uint4 zq[4];
+            if (!kSparse) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-              zq[i] = *reinterpret_cast<const uint4*>(zrow + ((static_cast<uint32_t>(c * 4 + i) ^ swz) << 4));
+              for (int i = 0; i < 4; ++i)
+                zq[i] = *reinterpret_cast<const uint4*>(zrow + ((static_cast<uint32_t>(c * 4 + i) ^ swz) << 4));
+            }
             tmem_ld_wait();
             const int nvalid = p.V - col0;  // columns of this chunk inside the vocabulary
             float zt[32];
+            if (!kSparse) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const uint32_t w[4] = {zq[i].x, zq[i].y, zq[i].z, zq[i].w};
+              for (int i = 0; i < 4; ++i) {
+                const uint32_t w[4] = {zq[i].x, zq[i].y, zq[i].z, zq[i].w};
 #pragma unroll
-              for (int k = 0; k < 4; ++k) {
-                zt[8 * i + 2 * k] = fmaxf(bf16_lo(w[k]), kNegClamp);
-                zt[8 * i + 2 * k + 1] = fmaxf(bf16_hi(w[k]), kNegClamp);
+                for (int k = 0; k < 4; ++k) {
+                  zt[8 * i + 2 * k] = fmaxf(bf16_lo(w[k]), kNegClamp);
+                  zt[8 * i + 2 * k + 1] = fmaxf(bf16_hi(w[k]), kNegClamp);
+                }
               }
             }
-            if (kMode == kForward) {
+            if (kMode == kForward && kSparse) {
+              // student statistics only
+              if (nvalid > 0) {
+                float zs[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) zs[i] = (i < nvalid) ? __uint_as_float(acc[i]) : kNegClamp;
+                float cb = zs[0];
+#pragma unroll
+                for (int i = 1; i < 32; ++i) cb = fmaxf(cb, zs[i]);
+                cb *= p.scale2;
+                if (cb > m_b) {
+                  s_b *= ex2f(m_b - cb);
+                  if (!kTauIsOne) s_b1 *= ex2f((m_b - cb) * p.tau);
+                  m_b = cb;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                  const float tb = fmaf(zs[i], p.scale2, -m_b);
+                  s_b += ex2f(tb);
+                  if (!kTauIsOne) s_b1 += ex2f(tb * p.tau);
+                }
+              }
+            } else if (kMode == kForward) {
               if (nvalid > 0) {
                 float zs[32];
 #pragma unroll
@@ -370,23 +419,32 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
               // gradient tile: dO_S = coef * (p_S - p_T), written back in place over the teacher
               uint32_t packed[16];
               const int yi = kComposite ? g_y - col0 : -1;  // label's place in this chunk, if any
+              float g[32];
 #pragma unroll
-              for (int i = 0; i < 32; i += 2) {
-                const float s0 = __uint_as_float(acc[i]), s1 = __uint_as_float(acc[i + 1]);
-                const float ps0 = ex2f(fmaf(s0, p.scale2, -g_lse_b)), ps1 = ex2f(fmaf(s1, p.scale2, -g_lse_b));
-                float g0 = g_coef * (ps0 - ex2f(fmaf(zt[i], p.scale2, -g_lse_a)));
-                float g1 = g_coef * (ps1 - ex2f(fmaf(zt[i + 1], p.scale2, -g_lse_a)));
+              for (int i = 0; i < 32; ++i) {
+                const float si = __uint_as_float(acc[i]);
+                const float ps = ex2f(fmaf(si, p.scale2, -g_lse_b));
+                g[i] = kSparse ? g_coef * ps : g_coef * (ps - ex2f(fmaf(zt[i], p.scale2, -g_lse_a)));
                 if (kComposite) {
                   // at temperature 1 the two student softmaxes are the same
-                  const float q0 = kTauIsOne ? ps0 : ex2f(fmaf(s0, 1.4426950408889634f, -g_lse_b1));
-                  const float q1 = kTauIsOne ? ps1 : ex2f(fmaf(s1, 1.4426950408889634f, -g_lse_b1));
-                  g0 = fmaf(g_cce, q0 - (i == yi ? 1.f : 0.f), g0);
-                  g1 = fmaf(g_cce, q1 - (i + 1 == yi ? 1.f : 0.f), g1);
+                  const float q = kTauIsOne ? ps : ex2f(fmaf(si, 1.4426950408889634f, -g_lse_b1));
+                  g[i] = fmaf(g_cce, q - (i == yi ? 1.f : 0.f), g[i]);
                 }
-                if (i >= nvalid) g0 = 0.f;
-                if (i + 1 >= nvalid) g1 = 0.f;
-                packed[i >> 1] = pack_bf16x2(g0, g1);
               }
+              if (kSparse) {
+                // the stored teacher probabilities that fall into this chunk (rare)
+#pragma unroll
+                for (int j = 0; j < kMaxTopK; ++j) {
+                  const int dj = tki[j] - col0;
+                  if (static_cast<unsigned>(dj) < 32u) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) g[i] -= (i == dj) ? tkc[j] : 0.f;
+                  }
+                }
+              }
+#pragma unroll
+              for (int i = 0; i < 32; i += 2)
+                packed[i >> 1] = pack_bf16x2(i < nvalid ? g[i] : 0.f, i + 1 < nvalid ? g[i + 1] : 0.f);
 #pragma unroll
               for (int i = 0; i < 4; ++i)
                 *reinterpret_cast<uint4*>(zrow + ((static_cast<uint32_t>(c * 4 + i) ^ swz) << 4)) =
@@ -394,8 +452,10 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             }
           }
           if (kMode == kForward) {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(zempty0 + bi);
+            if (!kSparse) {
+              __syncwarp();
+              if (lane == 0) mbar_arrive(zempty0 + bi);
+            }
           } else {
             // hand the finished 128 x 64 gradient sub-tile to TMA, then recycle the stage
             fence_proxy_async_smem();
@@ -407,7 +467,11 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                 tma_store_commit();
                 tma_store_wait_read<0>();
               }
-              mbar_arrive(zempty0 + bi);
+              // dense teacher: the stage goes back to the teacher producer.  Top-k teacher: the
+              // two stages of a half simply alternate; this thread has seen the store's read
+              // finish before it joins the next sub-tile's barrier, which every writer of the
+              // sub-tile after that has to pass first.
+              if (!kSparse) mbar_arrive(zempty0 + bi);
             }
           }
         }

@@ -76,7 +76,7 @@ struct Plan {
   bool dh_direct;     // dH stored straight to the output (one chunk, no split-K); else fp32 atomics
   bool grads;
   size_t off_status, off_plan, off_list, off_partials, off_lse_a, off_lse_b, off_coef, off_coef_ce,
-      off_lse_b1, off_g, off_dh, total;
+      off_lse_b1, off_tkcp, off_g, off_dh, total;
 };
 
 int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
@@ -132,6 +132,8 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
     pl->off_lse_b1 = off;
     off = align_up(off + sizeof(float) * a->T, 1024);
   }
+  pl->off_tkcp = off;
+  if (a->topk > 0) off = align_up(off + sizeof(float) * static_cast<size_t>(a->T) * a->topk, 1024);
   pl->off_g = off;
   pl->off_dh = off;
   if (pl->grads) {
@@ -152,9 +154,12 @@ int check_args(const npd_kd_args* a, bool need_pointers) {
   if (a->d_weight_dtype != NPD_DTYPE_BF16 && a->d_weight_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
   if (a->grad_chunk_cols < 0 || a->n_phase_events < 0) return NPD_EINVAL;
   if (a->d % 64 != 0) return NPD_ESHAPE;
-  if (a->ldh < a->d || a->ldw < a->d || a->ldt < a->V) return NPD_ESHAPE;
+  const bool sparse = a->topk != 0;
+  if (sparse && (a->topk < 0 || a->nll_teacher != nullptr)) return NPD_EINVAL;
+  if (sparse && a->topk > kd_cfg::kMaxTopK) return NPD_EUNSUPPORTED;
+  if (a->ldh < a->d || a->ldw < a->d || (!sparse && a->ldt < a->V)) return NPD_ESHAPE;
   if (a->cu_seqlens != nullptr && (a->S < 1 || a->S > a->T)) return NPD_ESHAPE;
-  if ((a->ldh % 8) || (a->ldw % 8) || (a->ldt % 8)) return NPD_EALIGN;
+  if ((a->ldh % 8) || (a->ldw % 8) || (!sparse && (a->ldt % 8))) return NPD_EALIGN;
   if ((a->d_hidden == nullptr) != (a->d_weight == nullptr)) return NPD_EINVAL;
   if ((a->flags & NPD_KD_ACCUMULATE_DW) && a->d_weight_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
   if (a->flags & NPD_KD_COMPOSITE_LOSS) {
@@ -162,9 +167,10 @@ int check_args(const npd_kd_args* a, bool need_pointers) {
     if (need_pointers && a->labels == nullptr) return NPD_EINVAL;
   }
   if (!need_pointers) return NPD_OK;
-  if (a->hidden == nullptr || a->weight == nullptr || a->teacher == nullptr || a->kl == nullptr)
+  if (a->hidden == nullptr || a->weight == nullptr || a->kl == nullptr) return NPD_EINVAL;
+  if (sparse ? (a->topk_values == nullptr || a->topk_indices == nullptr) : (a->teacher == nullptr))
     return NPD_EINVAL;
-  if (!aligned16(a->hidden) || !aligned16(a->weight) || !aligned16(a->teacher) ||
+  if (!aligned16(a->hidden) || !aligned16(a->weight) || (!sparse && !aligned16(a->teacher)) ||
       !aligned16(a->d_hidden) || !aligned16(a->d_weight))
     return NPD_EALIGN;
   if (a->d_weight != nullptr && a->d_weight_dtype == NPD_DTYPE_F32 && (a->ldw % 4)) return NPD_EALIGN;
@@ -240,12 +246,18 @@ int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const
 }
 
 template <int kMode>
-int launch_kd_tile(bool tau_one, bool composite, const CUtensorMap& mh, const CUtensorMap& mw, const CUtensorMap& mt,
+int launch_kd_tile(bool tau_one, bool composite, bool sparse, const CUtensorMap& mh, const CUtensorMap& mw, const CUtensorMap& mt,
                    const CUtensorMap& mg, const KdTileParams& kp, int sms, cudaStream_t st) {
   using namespace kd_cfg;
-  auto k = tau_one ? kd_tile_kernel<kMode, true, false> : kd_tile_kernel<kMode, false, false>;
-  if (kMode == kGradient && composite)
-    k = tau_one ? kd_tile_kernel<kMode, true, true> : kd_tile_kernel<kMode, false, true>;
+  composite = composite && kMode == kGradient;  // the forward does not depend on the objective's mix
+  auto k = kd_tile_kernel<kMode, true, false, false>;
+  if (!sparse) {
+    if (!composite) k = tau_one ? kd_tile_kernel<kMode, true, false, false> : kd_tile_kernel<kMode, false, false, false>;
+    else k = tau_one ? kd_tile_kernel<kMode, true, true, false> : kd_tile_kernel<kMode, false, true, false>;
+  } else {
+    if (!composite) k = tau_one ? kd_tile_kernel<kMode, true, false, true> : kd_tile_kernel<kMode, false, false, true>;
+    else k = tau_one ? kd_tile_kernel<kMode, true, true, true> : kd_tile_kernel<kMode, false, true, true>;
+  }
   if (set_smem(k, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
   // the number of units is only known on the device: always one CTA pair per two SMs
   const int grid = 2 * std::max(sms / 2, 1);
@@ -318,11 +330,17 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   const bool tau_one = a->temperature == 1.0f;
   const float scale2 = 1.4426950408889634f / a->temperature;
 
+  const bool sparse = a->topk > 0;  // teacher stored as its top-k logits per token
+  float* tk_cp = reinterpret_cast<float*>(ws + pl.off_tkcp);
   CUtensorMap mh, mw, mt;
   if (!make_map(&mh, a->hidden, a->d, a->T, a->ldh, 64, 128) ||
-      !make_map(&mw, a->weight, a->d, a->V, a->ldw, 64, 128) ||
-      !make_map(&mt, a->teacher, a->V, a->T, a->ldt, 64, 128))
+      !make_map(&mw, a->weight, a->d, a->V, a->ldw, 64, 128))
     return NPD_ECUDA;
+  if (sparse) {
+    mt = mh;  // never used: no teacher tiles are streamed
+  } else if (!make_map(&mt, a->teacher, a->V, a->T, a->ldt, 64, 128)) {
+    return NPD_ECUDA;
+  }
 
   // cu_seqlens is validated on the device; the result lands in the status word.
   if (a->cu_seqlens != nullptr) {
@@ -361,9 +379,41 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   kp.tau = a->temperature;
   kp.partials = partials;
   kp.status = status;
-  if ((rc = launch_kd_tile<kForward>(tau_one, false, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
+  if ((rc = launch_kd_tile<kForward>(tau_one, false, sparse, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
   rec.mark();
 
+  if (sparse) {
+    CombineTopkParams tp{};
+    tp.T = a->T;
+    tp.d = a->d;
+    tp.V = a->V;
+    tp.topk = a->topk;
+    tp.plan = plan;
+    tp.partials = partials;
+    tp.hidden = static_cast<const __nv_bfloat16*>(a->hidden);
+    tp.weight = static_cast<const __nv_bfloat16*>(a->weight);
+    tp.ldh = a->ldh;
+    tp.ldw = a->ldw;
+    tp.tk_val = a->topk_values;
+    tp.tk_idx = a->topk_indices;
+    tp.loss_mask = a->loss_mask;
+    tp.labels = a->labels;
+    tp.scale2 = scale2;
+    tp.tau = a->temperature;
+    tp.grad_scale = a->grad_scale;
+    tp.lambda = composite ? a->kd_lambda : 1.f;
+    tp.kl = a->kl;
+    tp.nll_s = a->nll_student;
+    tp.lse2_b = lse_b;
+    tp.coef = coef;
+    tp.tk_cp = tk_cp;
+    tp.coef_ce = coef_ce;
+    tp.lse2_b1 = lse_b1;
+    if (tau_one)
+      kd_combine_topk_kernel<true><<<(a->T + 7) / 8, 256, 0, st>>>(tp);
+    else
+      kd_combine_topk_kernel<false><<<(a->T + 7) / 8, 256, 0, st>>>(tp);
+  }
   CombineParams cp{};
   cp.T = a->T;
   cp.d = a->d;
@@ -390,10 +440,13 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   cp.lambda = composite ? a->kd_lambda : 1.f;
   cp.coef_ce = coef_ce;
   cp.lse2_b1 = lse_b1;
-  if (tau_one)
+  if (sparse) {
+    // merged above
+  } else if (tau_one) {
     kd_combine_kernel<true><<<(a->T + 7) / 8, 256, 0, st>>>(cp);
-  else
+  } else {
     kd_combine_kernel<false><<<(a->T + 7) / 8, 256, 0, st>>>(cp);
+  }
   ++g_launches;
   if (cudaGetLastError() != cudaSuccess) return NPD_ECUDA;
   rec.mark();
@@ -430,8 +483,11 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     gp.coef_ce = coef_ce;
     gp.lse2_b1 = lse_b1;
     gp.labels = a->labels;
+    gp.tk_idx = a->topk_indices;
+    gp.tk_cp = tk_cp;
+    gp.topk = a->topk;
     gp.g_col0 = col0;
-    if ((rc = launch_kd_tile<kGradient>(tau_one, composite, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
+    if ((rc = launch_kd_tile<kGradient>(tau_one, composite, sparse, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
     rec.mark();
 
     GemmProblem pr[2] = {};
@@ -510,14 +566,25 @@ int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* c
   int rc = check_args(dev, true);
   if (rc != NPD_OK) return rc;
   if (host->T != dev->T || host->d != dev->d || host->V != dev->V) return NPD_EINVAL;
-  if (host->hidden == nullptr || host->teacher == nullptr || host->kl == nullptr) return NPD_EINVAL;
+  if (host->hidden == nullptr || host->kl == nullptr || host->topk != dev->topk) return NPD_EINVAL;
+  if (dev->topk > 0 ? (host->topk_values == nullptr || host->topk_indices == nullptr)
+                    : (host->teacher == nullptr))
+    return NPD_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t T = dev->T;
   bool ok = true;
   ok &= cudaMemcpy2DAsync(const_cast<void*>(dev->hidden), dev->ldh * 2, host->hidden, host->ldh * 2,
                           static_cast<size_t>(dev->d) * 2, T, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpy2DAsync(const_cast<void*>(dev->teacher), dev->ldt * 2, host->teacher, host->ldt * 2,
-                          static_cast<size_t>(dev->V) * 2, T, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (dev->topk > 0) {
+    const size_t n = T * static_cast<size_t>(dev->topk);
+    ok &= cudaMemcpyAsync(const_cast<float*>(dev->topk_values), host->topk_values, n * sizeof(float),
+                          cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->topk_indices), host->topk_indices, n * sizeof(int32_t),
+                          cudaMemcpyHostToDevice, st) == cudaSuccess;
+  } else {
+    ok &= cudaMemcpy2DAsync(const_cast<void*>(dev->teacher), dev->ldt * 2, host->teacher, host->ldt * 2,
+                            static_cast<size_t>(dev->V) * 2, T, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
   if (dev->cu_seqlens != nullptr && host->cu_seqlens != nullptr)
     ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->cu_seqlens), host->cu_seqlens,
                           sizeof(int32_t) * (dev->S + 1), cudaMemcpyHostToDevice, st) == cudaSuccess;

@@ -226,6 +226,131 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
   }
 }
 
+struct CombineTopkParams {
+  int T, d, V, topk;
+  const int* plan;        // plan[2] = forward runs; the partials hold 2 slots per run
+  const float* partials;  // [2*runs][kPFields][T]; only the student's fields are filled
+  const __nv_bfloat16* hidden;
+  const __nv_bfloat16* weight;
+  long long ldh, ldw;
+  const float* tk_val;    // [T, topk] stored teacher logits
+  const int32_t* tk_idx;  // [T, topk] their vocabulary indices
+  const uint8_t* loss_mask;
+  const int32_t* labels;
+  float scale2, tau, grad_scale, lambda;
+  float* kl;
+  float* nll_s;
+  float* lse2_b;
+  float* coef;
+  float* tk_cp;           // [T, topk] coef_t * p_T(j), for the gradient tiles
+  float* coef_ce;         // composite objective only (else NULL)
+  float* lse2_b1;
+};
+
+// <H[t], W[c]> in fp32, one warp.
+__device__ __forceinline__ float warp_dot_bf16(const __nv_bfloat16* h, const __nv_bfloat16* w, int d, int lane) {
+  const uint4* h4 = reinterpret_cast<const uint4*>(h);
+  const uint4* w4 = reinterpret_cast<const uint4*>(w);
+  float dot = 0.f;
+  for (int i = lane; i < d / 8; i += 32) {
+    const uint4 a = h4[i], b = w4[i];
+    dot = fmaf(bf16_lo(a.x), bf16_lo(b.x), dot);
+    dot = fmaf(bf16_hi(a.x), bf16_hi(b.x), dot);
+    dot = fmaf(bf16_lo(a.y), bf16_lo(b.y), dot);
+    dot = fmaf(bf16_hi(a.y), bf16_hi(b.y), dot);
+    dot = fmaf(bf16_lo(a.z), bf16_lo(b.z), dot);
+    dot = fmaf(bf16_hi(a.z), bf16_hi(b.z), dot);
+    dot = fmaf(bf16_lo(a.w), bf16_lo(b.w), dot);
+    dot = fmaf(bf16_hi(a.w), bf16_hi(b.w), dot);
+  }
+  return warp_sum(dot);
+}
+
+// One warp per token, teacher stored as its k largest logits (Eq. 2 as printed).  Merges the
+// student's partials into lse(O_S/tau), forms p_T = Softmax of the k stored logits / tau, takes
+// the student logit at each stored index as the dot product <H[t], W[idx]> in fp32, and sums
+//   KL = sum_j p_T(j) (log p_T(j) - (O_S[idx_j]/tau - lse)).
+template <bool kTauIsOne>
+__global__ void __launch_bounds__(256) kd_combine_topk_kernel(const CombineTopkParams p) {
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= p.T) return;
+  const bool on = p.loss_mask == nullptr || p.loss_mask[t] != 0;
+  float* cp = p.tk_cp + static_cast<size_t>(t) * p.topk;
+  if (!on) {
+    if (lane == 0) {
+      p.kl[t] = 0.f;
+      if (p.nll_s != nullptr) p.nll_s[t] = 0.f;
+      p.lse2_b[t] = 1e30f;
+      p.coef[t] = 0.f;
+      if (p.coef_ce != nullptr) {
+        p.coef_ce[t] = 0.f;
+        p.lse2_b1[t] = 1e30f;
+      }
+    }
+    for (int j = lane; j < p.topk; j += 32) cp[j] = 0.f;
+    return;
+  }
+  const int nslots = 2 * p.plan[2];
+  const size_t fs = static_cast<size_t>(p.T), ss = static_cast<size_t>(kPFields) * fs;
+  float mb = -INFINITY;
+  for (int s = lane; s < nslots; s += 32) mb = fmaxf(mb, p.partials[s * ss + kPMaxB * fs + t]);
+  mb = warp_max(mb);
+  float sb = 0.f, sb1 = 0.f;
+  for (int s = lane; s < nslots; s += 32) {
+    const float* q = p.partials + s * ss + t;
+    const float db = q[kPMaxB * fs] - mb;
+    sb = fmaf(q[kPSumB * fs], exp2f(db), sb);
+    if (!kTauIsOne) sb1 = fmaf(q[kPSumB1 * fs], exp2f(db * p.tau), sb1);
+  }
+  sb = warp_sum(sb);
+  if (!kTauIsOne) sb1 = warp_sum(sb1);
+  const float lse_b = mb + log2f(sb);                    // base 2, of O_S * log2(e)/tau
+  const float lse_b1 = kTauIsOne ? lse_b : mb * p.tau + log2f(sb1);  // same at temperature 1
+  const __nv_bfloat16* h = p.hidden + static_cast<size_t>(t) * p.ldh;
+
+  // teacher distribution on its stored support (lane j holds entry j; topk <= 32)
+  const float v = lane < p.topk ? p.tk_val[static_cast<size_t>(t) * p.topk + lane] : -INFINITY;
+  const float a2 = fmaxf(v, kd_cfg::kNegClamp) * p.scale2;       // base-2 scaled teacher logit
+  const float ma = warp_max(lane < p.topk ? a2 : -INFINITY);
+  const float ea = lane < p.topk ? exp2f(a2 - ma) : 0.f;
+  const float sa = warp_sum(ea);
+  const float pt = ea / sa;
+  const float lse_a = ma + log2f(sa);
+  float kl = 0.f;
+  for (int j = 0; j < p.topk; ++j) {
+    int c = p.tk_idx[static_cast<size_t>(t) * p.topk + j];
+    c = c < 0 ? 0 : (c >= p.V ? p.V - 1 : c);               // indices outside [0,V) are a caller error
+    const float sj = warp_dot_bf16(h, p.weight + static_cast<size_t>(c) * p.ldw, p.d, lane);
+    const float ptj = __shfl_sync(0xffffffffu, pt, j), a2j = __shfl_sync(0xffffffffu, a2, j);
+    // log2 p_T(j) - log2 p_S(idx_j); a zero probability contributes nothing
+    if (ptj > 0.f) kl = fmaf(ptj, (a2j - lse_a) - (sj * p.scale2 - lse_b), kl);
+  }
+  float nll_s = 0.f;
+  bool has_label = false;
+  if (p.labels != nullptr) {
+    const int y = p.labels[t];
+    if (y >= 0 && y < p.V) {
+      has_label = true;
+      const float dot = warp_dot_bf16(h, p.weight + static_cast<size_t>(y) * p.ldw, p.d, lane);
+      nll_s = kLn2 * lse_b1 - dot;
+    }
+  }
+  const float coef = p.grad_scale * p.lambda / p.tau;
+  if (lane < p.topk) cp[lane] = coef * pt;
+  if (lane == 0) {
+    kl *= kLn2;
+    p.kl[t] = kl < 0.f ? 0.f : kl;
+    if (p.nll_s != nullptr) p.nll_s[t] = nll_s;
+    p.lse2_b[t] = lse_b;
+    p.coef[t] = coef;
+    if (p.coef_ce != nullptr) {
+      p.coef_ce[t] = has_label ? p.grad_scale * (1.f - p.lambda) : 0.f;
+      p.lse2_b1[t] = lse_b1;
+    }
+  }
+}
+
 // One warp per packed segment: masked sums of the per-token values and the count of
 // tokens that carry a label, reduced with warp shuffles in a fixed order; also the
 // token -> segment map and the validation of cu_seqlens.

@@ -77,6 +77,30 @@ def test_config2_full_size_sampled_rows_and_dweight_rows():
     assert frob(got, ref) <= GRAD_FROB
 
 
+def test_config2_full_size_top_k_teacher_sampled_rows():
+    # the paper's storage form: k = 10 teacher logits per token, composite objective with lambda = 0.9
+    b = syn.config2_1b(device=DEV)
+    vals, idx = b.teacher.float().topk(10, dim=1)
+    idx = idx.to(torch.int32).contiguous()
+    vals = vals.contiguous()
+    step = run_step(b, topk_values=vals, topk_indices=idx, kd_lambda=0.9)
+    rows = _sample_rows(b, 40, 5)
+    r = torch.from_numpy(rows).to(DEV)
+    W = host(b.weight)
+    H, v, i = host(b.hidden[r]), host(vals[r]), idx[r].cpu().numpy()
+    y, m = b.labels[r].cpu().numpy(), b.loss_mask[r].cpu().numpy()
+    kl, ns = orc.topk_kd_token_losses(H, W, v, i, y, m, b.tau)
+    assert_losses_close(host(step.kl[r]), kl, "kl rows")
+    assert_losses_close(host(step.nll_student[r]), ns, "nll_student rows")
+    dense = np.full((len(rows), b.V), -np.inf)
+    np.put_along_axis(dense, i.astype(np.int64), v, axis=1)
+    dO = orc.composite_logit_gradient(H, W, dense, y, m, b.tau, step.grad_scale, 0.9)
+    assert frob(host(step.d_hidden[r]), dO @ W) <= GRAD_FROB
+    mm = b.loss_mask.bool()
+    assert float(step.kl[~mm].abs().max()) == 0.0 and float(step.d_hidden[~mm].float().abs().max()) == 0.0
+    assert bool(torch.isfinite(step.d_weight.float()).all())
+
+
 def test_config3_full_size_sampled_rows_temperature_two():
     b = syn.config3_rows(device=DEV)
     assert (b.T, b.d, b.tau) == (32768, 2048, 2.0)

@@ -124,6 +124,65 @@ def test_composite_objective_gradients(tau, lam):
         assert torch.equal(plain.d_weight, step.d_weight)
 
 
+def _topk_of(b, k):
+    """The k largest teacher logits per token and their indices, as the annotation phase stores them."""
+    vals, idx = b.teacher.float().topk(k, dim=1)
+    return vals.contiguous(), idx.to(torch.int32).contiguous()
+
+
+@pytest.mark.parametrize("tau,k,lam", [(1.0, 10, None), (2.0, 4, None), (1.0, 16, 0.9), (1.3, 1, 0.5)])
+def test_topk_teacher_matches_the_oracle(tau, k, lam):
+    # Eq. 2 as printed: the teacher is its k largest logits per token
+    b = syn.scaled("c2", device=DEV, T=700, d=128, V=3000, min_len=20, max_len=300)
+    b.tau = tau
+    vals, idx = _topk_of(b, k)
+    step = run_step(b, topk_values=vals, topk_indices=idx, kd_lambda=lam, dw_dtype=torch.float32,
+                    grad_chunk_cols=1024)
+    H, W, Z, y, m = oracle_inputs(b)
+    v, i = host(vals), idx.cpu().numpy()
+    kl, ns = orc.topk_kd_token_losses(H, W, v, i, y, m, tau)
+    assert_losses_close(host(step.kl), kl, "kl")
+    assert_losses_close(host(step.nll_student), ns, "nll_student")
+    if lam is None:
+        dH, dW = orc.topk_kd_backward(H, W, v, i, m, tau, step.grad_scale)
+    else:   # composite objective with the top-k distillation term: same Eq. 1, dense form with -inf fill
+        dense = np.full_like(Z, -np.inf)
+        np.put_along_axis(dense, i.astype(np.int64), v, axis=1)
+        dH, dW = orc.composite_backward(H, W, dense, y, m, tau, step.grad_scale, lam)
+    assert frob(host(step.d_hidden), dH) <= GRAD_FROB
+    assert frob(host(step.d_weight), dW) <= GRAD_FROB
+    assert np.all(host(step.d_hidden)[m == 0] == 0) and np.all(host(step.kl)[m == 0] == 0)
+
+
+def test_topk_teacher_equals_dense_teacher_with_minus_inf_fill():
+    # the two entry forms of the same teacher agree on the GPU as well
+    b = syn.scaled("c2", device=DEV, T=300, d=64, V=1000, min_len=20, max_len=90)
+    vals, idx = _topk_of(b, 10)
+    sparse = run_step(b, topk_values=vals, topk_indices=idx, dw_dtype=torch.float32)
+    dense = torch.full_like(b.teacher, float("-inf"))
+    dense.scatter_(1, idx.long(), vals.to(torch.bfloat16))
+    b.teacher = dense
+    full = run_step(b, dw_dtype=torch.float32)
+    assert_losses_close(host(sparse.kl), host(full.kl), "kl")
+    assert frob(host(sparse.d_weight), host(full.d_weight)) < 5e-3
+    assert frob(host(sparse.d_hidden), host(full.d_hidden)) < 1e-2
+
+
+def test_topk_teacher_argument_errors():
+    b = _mini()
+    vals, idx = _topk_of(b, 4)
+    step = B.KDStep(b, topk_values=vals, topk_indices=idx)
+    a = B.npd_kd_args.from_buffer_copy(step.args)
+    a.topk = 17
+    assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EUNSUPPORTED
+    a = B.npd_kd_args.from_buffer_copy(step.args)
+    a.topk_indices = None
+    assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EINVAL
+    a = B.npd_kd_args.from_buffer_copy(step.args)
+    a.nll_teacher = step.kl.data_ptr()
+    assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EINVAL
+
+
 def test_runs_are_bitwise_reproducible():
     b = syn.scaled("c2", device=DEV, T=700, d=128, V=3000, min_len=20, max_len=300)
     s1 = run_step(b, grad_chunk_cols=1024)
