@@ -61,6 +61,7 @@ __all__ = [
     "validate_cu_seqlens",
     "segment_ids",
     "segment_stats",
+    "reverse_kl_token",
     "ifd_scores",
     "delta_ifd_select",
     "nearest_rank_percentile",
@@ -186,6 +187,30 @@ def kd_dweight_rows(H, W, teacher_logits, loss_mask, tau, grad_scale, vocab_rows
         dO = kd_logit_gradient(Hg, W, Zg, np.asarray(loss_mask[t0:t1]), tau, grad_scale)
         out += np.matmul(dO[:, c].T, Hg)
     return out
+
+
+# --------------------------------------------------------------------------- #
+# Policy-lag monitor (appendix, "Analysis of Policy Latency")
+# --------------------------------------------------------------------------- #
+
+def reverse_kl_token(H, W, generator_logits, loss_mask, tau: float = 1.0):
+    """Per-token D_KL(pi_learner || pi_generator), the quantity the appendix tracks to bound
+    the policy lag:  the learner is the current student, p_L = Softmax(H W^T / tau), the
+    generator's logits for the same positions are given;
+
+        rkl[t] = m_t * sum_c p_L(c) (log p_L(c) - log p_G(c)).
+
+    Note the direction: the learner's distribution weighs the sum (Eq. 2 has the teacher's)."""
+    O_L = student_logits(H, W)
+    O_G = _f64(generator_logits)[:, : O_L.shape[1]]
+    logp_L = log_softmax(O_L / tau)
+    logp_G = log_softmax(O_G / tau)
+    p_L = np.exp(logp_L)
+    with np.errstate(invalid="ignore"):
+        terms = p_L * (logp_L - logp_G)
+    terms = np.where(p_L > 0.0, terms, 0.0)
+    m = np.asarray(loss_mask).astype(bool)
+    return np.where(m, terms.sum(axis=1), 0.0)
 
 
 # --------------------------------------------------------------------------- #
@@ -370,7 +395,8 @@ def ifd_scores(cond_seg, uncond_seg, nll_sum, count, dtype=np.float64):
 
 def delta_ifd_select(cond_seg, uncond_seg, nll_s_sum, nll_t_sum, count,
                      lo: float, hi: float, require_teacher_ifd_le_1: bool = False,
-                     dtype=np.float64):
+                     dtype=np.float64, score: str = "delta", lo_inclusive: bool = True,
+                     hi_inclusive: bool = True):
     """Delta_IFD = IFD_Teacher - IFD_Student  (Eq. 4) and the keep rule of the
     Proximal Learning Zone:  keep iff lo <= Delta <= hi (both ends inclusive;
     the paper's lo is 0 and hi its difficulty threshold).  Delta < lo is the
@@ -378,17 +404,25 @@ def delta_ifd_select(cond_seg, uncond_seg, nll_s_sum, nll_t_sum, count,
     extra condition IFD_Teacher <= 1 is the "teacher confirms base quality"
     remark of the zone description.  NaN scores are never kept.
 
+    The filter ablation (the table of filtering metrics and selection scopes) tests the
+    same interval rule on other scores and with open ends: ``score`` picks what is
+    tested ("delta", "ifd_teacher" or "ifd_student"), ``lo_inclusive`` / ``hi_inclusive``
+    say whether an end belongs to the scope; an infinite end leaves that side open-ended.
+
     Returns (ifd_teacher, ifd_student, delta, keep uint8, n_keep int).
     """
     ifd_t = ifd_scores(cond_seg, uncond_seg, nll_t_sum, count, dtype)
     ifd_s = ifd_scores(cond_seg, uncond_seg, nll_s_sum, count, dtype)
     delta = (ifd_t - ifd_s).astype(dtype)
     f = np.dtype(dtype).type
+    tested = {"delta": delta, "ifd_teacher": ifd_t, "ifd_student": ifd_s}[score]
     with np.errstate(invalid="ignore"):
-        keep = (delta >= f(lo)) & (delta <= f(hi))
+        above = (tested >= f(lo)) if lo_inclusive else (tested > f(lo))
+        below = (tested <= f(hi)) if hi_inclusive else (tested < f(hi))
+        keep = above & below
         if require_teacher_ifd_le_1:
             keep &= ifd_t <= f(1.0)
-    keep &= ~np.isnan(delta)
+    keep &= ~np.isnan(tested)
     return ifd_t, ifd_s, delta, keep.astype(np.uint8), int(keep.sum())
 
 

@@ -169,3 +169,52 @@ def test_nearest_rank_percentile():
     assert orc.nearest_rank_percentile([5, 1, 3, 2, 4], 0.81) == 5
     assert orc.nearest_rank_percentile([1, float("nan"), 2, 3, 4, 5], 0.2) == 1
     assert orc.nearest_rank_percentile(np.arange(1, 11), 0.8) == 8
+
+
+def test_filter_ablation_scopes_on_the_hand_worked_table():
+    rows = _read_golden()
+    n = len(rows)
+    count = np.zeros(2 * n, dtype=np.int32)
+    t_sum, s_sum = np.zeros(2 * n), np.zeros(2 * n)
+    for i, r in enumerate(rows):
+        count[2 * i], count[2 * i + 1] = r["cc"], r["cu"]
+        t_sum[2 * i], t_sum[2 * i + 1] = r["tc"], r["tu"]
+        s_sum[2 * i], s_sum[2 * i + 1] = r["sc"], r["su"]
+    cond = np.arange(n) * 2
+    unc = cond + 1
+    want = []
+    path = os.path.join(os.path.dirname(__file__), "golden", "filter_variants_table.txt")
+    for line in open(path):
+        if line.strip() and not line.startswith("#"):
+            want.append([int(x) for x in line.split("|")[1].split()])
+    want = np.asarray(want)
+    inf = float("inf")
+    variants = [dict(score="ifd_teacher", lo=0.0, hi=1.0), dict(score="ifd_student", lo=0.0, hi=1.0),
+                dict(score="delta", lo=0.0, hi=inf, lo_inclusive=False),
+                dict(score="delta", lo=-inf, hi=1.0, hi_inclusive=False),
+                dict(score="delta", lo=0.0, hi=1.0)]
+    for col, v in enumerate(variants):
+        for dtype in (np.float64, np.float32):
+            keep = orc.delta_ifd_select(cond, unc, s_sum, t_sum, count, dtype=dtype, **v)[3]
+            assert keep.tolist() == want[:, col].tolist(), v
+
+
+def test_reverse_kl_is_the_forward_kl_with_the_roles_swapped():
+    # D(learner || generator) computed by the monitor = Eq. 2's divergence with the learner's
+    # logits in the teacher's seat and the generator's logits produced by an identity head
+    rng = np.random.default_rng(9)
+    T, d, V = 7, 5, 6
+    H, W = rng.standard_normal((T, d)), rng.standard_normal((V, d))
+    G = rng.standard_normal((T, V)) * 2
+    m = np.array([1, 0, 1, 1, 1, 0, 1], dtype=np.uint8)
+    for tau in (1.0, 1.7):
+        rkl = orc.reverse_kl_token(H, W, G, m, tau)
+        swapped, _, _ = orc.kd_token_losses(G, np.eye(V), H @ W.T, np.full(T, -1), m, tau)
+        assert np.allclose(rkl, swapped, atol=1e-13)
+        assert np.all(rkl >= 0) and np.all(rkl[m == 0] == 0)
+    assert np.abs(orc.reverse_kl_token(H, W, H @ W.T + 3.0, m)).max() < 1e-12   # same policy, shifted logits
+    fwd, _, _ = orc.kd_token_losses(H, W, G, np.full(T, -1), m, 1.0)
+    assert not np.allclose(fwd, orc.reverse_kl_token(H, W, G, m))              # the direction matters
+    from scipy.special import rel_entr, softmax
+    ref = rel_entr(softmax(H @ W.T, axis=1), softmax(G, axis=1)).sum(axis=1) * m
+    assert np.allclose(orc.reverse_kl_token(H, W, G, m), ref, atol=1e-13)
