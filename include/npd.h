@@ -63,7 +63,7 @@ enum { NPD_DTYPE_BF16 = 0, NPD_DTYPE_F32 = 1 };
 /* flags of npd_kd_args */
 enum {
   NPD_KD_ACCUMULATE_DW = 1, /* add into d_weight instead of overwriting it (f32 d_weight only) */
-  NPD_KD_COMPOSITE_LOSS = 2 /* gradients of the composite objective of Eq. 1,
+  NPD_KD_COMPOSITE_LOSS = 2,/* gradients of the composite objective of Eq. 1,
                                L_total = (1 - lambda) L_CE + lambda L_KD with lambda = kd_lambda:
                                  dO_S[t,c] = grad_scale * m_t * ( lambda (p_S - p_T) / tau
                                              + (1 - lambda) [y_t>=0] (Softmax(O_S[t])[c] - [c = y_t]) )
@@ -71,6 +71,11 @@ enum {
                                outputs are unchanged: the loss value of a token is
                                (1 - lambda) * nll_student[t] + lambda * kl[t].  Without the flag
                                the gradients are those of Eq. 2 alone (lambda = 1). */
+  NPD_KD_REVERSE_KL = 4     /* forward only (d_hidden, d_weight NULL; dense `teacher`): kl[t] becomes
+                               m_t * D_KL(p_S || p_G) = sum_c p_S(c) (log p_S(c) - log p_G(c)) with
+                               p_G = Softmax(teacher[t]/tau), i.e. the divergence of the current
+                               learner from the logits of the policy that generated the data, which
+                               the paper's appendix tracks as policy lag.  Needs finite logits. */
 };
 
 /*
@@ -192,7 +197,13 @@ int npd_segment_stats(int32_t T, int32_t S, const int32_t* cu_seqlens,
 
 /* flags of npd_select */
 enum {
-  NPD_SELECT_TEACHER_IFD_LE_1 = 1 /* also require IFD_Teacher <= 1 (Section 3.2, zone text) */
+  NPD_SELECT_TEACHER_IFD_LE_1 = 1,  /* also require IFD_Teacher <= 1 (Section 3.2, zone text) */
+  /* the selection scopes of the paper's filter ablation: the interval tests another score,
+     or has open ends (an infinite lo / hi leaves that side unbounded) */
+  NPD_SELECT_SCORE_IFD_TEACHER = 2, /* keep = lo <= ifd_teacher <= hi */
+  NPD_SELECT_SCORE_IFD_STUDENT = 4, /* keep = lo <= ifd_student <= hi */
+  NPD_SELECT_LO_EXCLUSIVE = 8,      /* lo <  score */
+  NPD_SELECT_HI_EXCLUSIVE = 16      /* score <  hi */
 };
 
 /*

@@ -22,7 +22,10 @@ NPD_EWORKSPACE, NPD_ECUDA, NPD_ETIMEOUT, NPD_EUNSUPPORTED = -6, -7, -8, -9
 NPD_DTYPE_BF16, NPD_DTYPE_F32 = 0, 1
 NPD_KD_ACCUMULATE_DW = 1
 NPD_KD_COMPOSITE_LOSS = 2
+NPD_KD_REVERSE_KL = 4
 NPD_SELECT_TEACHER_IFD_LE_1 = 1
+NPD_SELECT_SCORE_IFD_TEACHER, NPD_SELECT_SCORE_IFD_STUDENT = 2, 4
+NPD_SELECT_LO_EXCLUSIVE, NPD_SELECT_HI_EXCLUSIVE = 8, 16
 NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32 = range(4)
 
 EXPORTS = ("npd_workspace_bytes", "npd_phase_count", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
@@ -236,7 +239,7 @@ class KDStep:
     fused step on them; a convenience over the raw calls."""
 
     def __init__(self, batch, *, grads=True, dw_dtype=torch.bfloat16, grad_chunk_cols=0, grad_scale=None,
-                 kd_lambda=None, topk_values=None, topk_indices=None):
+                 kd_lambda=None, topk_values=None, topk_indices=None, flags=0):
         dev = batch.hidden.device
         T, d, V = batch.T, batch.d, batch.V
         f32 = dict(dtype=torch.float32, device=dev)
@@ -255,7 +258,8 @@ class KDStep:
                         temperature=batch.tau, grad_scale=self.grad_scale, kl=self.kl,
                         nll_student=self.nll_student, nll_teacher=self.nll_teacher,
                         d_hidden=self.d_hidden, d_weight=self.d_weight, grad_chunk_cols=grad_chunk_cols,
-                        kd_lambda=kd_lambda, topk_values=topk_values, topk_indices=topk_indices)
+                        kd_lambda=kd_lambda, topk_values=topk_values, topk_indices=topk_indices,
+                        flags=flags)
         teacher = batch.teacher if topk_values is None else None
         probe = make_kd_args(batch.hidden, batch.weight, teacher, **self._kw)
         nbytes = npd_workspace_bytes(probe)

@@ -65,6 +65,8 @@ struct KdTileParams {
   float tau;
   // forward
   float* partials;  // [2*nsplit][kPFields][T]
+  int reverse;      // 1: the cross term is weighted by the student's probabilities (the divergence
+                    // of the policy-lag monitor, student || given logits) instead of the teacher's
   // gradient
   const float* lse2_a;  // [T] log2-sum-exp2 of the scaled teacher logits
   const float* lse2_b;  // [T] same for the student
@@ -389,15 +391,18 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                 for (int i = 1; i < 32; ++i) { ca = fmaxf(ca, zt[i]); cb = fmaxf(cb, zs[i]); }
                 ca *= p.scale2;
                 cb *= p.scale2;
+                const bool rev = p.reverse != 0;  // uniform over the grid
                 if (ca > m_a) {
                   const float f = ex2f(m_a - ca);
                   s_a *= f;
-                  cross *= f;
+                  if (!rev) cross *= f;
                   if (!kTauIsOne) s_a1 *= ex2f((m_a - ca) * p.tau);
                   m_a = ca;
                 }
                 if (cb > m_b) {
-                  s_b *= ex2f(m_b - cb);
+                  const float f = ex2f(m_b - cb);
+                  s_b *= f;
+                  if (rev) cross *= f;
                   if (!kTauIsOne) s_b1 *= ex2f((m_b - cb) * p.tau);
                   m_b = cb;
                 }
@@ -405,10 +410,10 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                 for (int i = 0; i < 32; ++i) {
                   const float ta = fmaf(zt[i], p.scale2, -m_a);
                   const float tb = fmaf(zs[i], p.scale2, -m_b);
-                  const float ea = ex2f(ta);
+                  const float ea = ex2f(ta), eb = ex2f(tb);
                   s_a += ea;
-                  cross = fmaf(ea, zt[i] - zs[i], cross);
-                  s_b += ex2f(tb);
+                  cross = fmaf(rev ? eb : ea, zt[i] - zs[i], cross);
+                  s_b += eb;
                   if (!kTauIsOne) {
                     s_a1 += ex2f(ta * p.tau);
                     s_b1 += ex2f(tb * p.tau);

@@ -162,6 +162,7 @@ int check_args(const npd_kd_args* a, bool need_pointers) {
   if ((a->ldh % 8) || (a->ldw % 8) || (!sparse && (a->ldt % 8))) return NPD_EALIGN;
   if ((a->d_hidden == nullptr) != (a->d_weight == nullptr)) return NPD_EINVAL;
   if ((a->flags & NPD_KD_ACCUMULATE_DW) && a->d_weight_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
+  if ((a->flags & NPD_KD_REVERSE_KL) && (a->d_hidden != nullptr || a->topk != 0)) return NPD_EINVAL;
   if (a->flags & NPD_KD_COMPOSITE_LOSS) {
     if (!(a->kd_lambda >= 0.f && a->kd_lambda <= 1.f)) return NPD_EINVAL;
     if (need_pointers && a->labels == nullptr) return NPD_EINVAL;
@@ -378,6 +379,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   kp.scale2 = scale2;
   kp.tau = a->temperature;
   kp.partials = partials;
+  kp.reverse = (a->flags & NPD_KD_REVERSE_KL) ? 1 : 0;
   kp.status = status;
   if ((rc = launch_kd_tile<kForward>(tau_one, false, sparse, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
   rec.mark();
@@ -438,6 +440,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   cp.lse2_b = lse_b;
   cp.coef = coef;
   cp.lambda = composite ? a->kd_lambda : 1.f;
+  cp.reverse = kp.reverse;
   cp.coef_ce = coef_ce;
   cp.lse2_b1 = lse_b1;
   if (sparse) {
@@ -630,6 +633,7 @@ int npd_select(int32_t N, const int32_t* cond_seg, const int32_t* uncond_seg, co
       nll_t_sum == nullptr || count == nullptr || keep == nullptr || n_keep == nullptr)
     return NPD_EINVAL;
   if (std::isnan(lo) || std::isnan(hi)) return NPD_EINVAL;
+  if ((flags & NPD_SELECT_SCORE_IFD_TEACHER) && (flags & NPD_SELECT_SCORE_IFD_STUDENT)) return NPD_EINVAL;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(n_keep, 0, sizeof(int32_t), st) != cudaSuccess) return NPD_ECUDA;
   select_kernel<<<(N + 255) / 256, 256, 0, st>>>(N, S, cond_seg, uncond_seg, nll_s_sum, nll_t_sum, count,

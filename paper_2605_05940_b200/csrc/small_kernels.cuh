@@ -119,6 +119,7 @@ struct CombineParams {
   float lambda;
   float* coef_ce;
   float* lse2_b1;
+  int reverse;  // 1: kl[t] = D(student || given logits), the cross partials carry the student's weights
 };
 
 // One warp per token.  Merges the per-split online-softmax partials into the token's
@@ -165,7 +166,7 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
     const float da = q[kPMaxA * fs] - ma, db = q[kPMaxB * fs] - mb;
     const float fa = exp2f(da), fb = exp2f(db);
     sa = fmaf(q[kPSumA * fs], fa, sa);
-    cr = fmaf(q[kPCross * fs], fa, cr);
+    cr = fmaf(q[kPCross * fs], p.reverse ? fb : fa, cr);
     sb = fmaf(q[kPSumB * fs], fb, sb);
     if (!kTauIsOne) {
       sa1 = fmaf(q[kPSumA1 * fs], exp2f(da * p.tau), sa1);
@@ -212,7 +213,9 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
     }
   }
   if (lane == 0) {
-    const float kl = kLn2 * (p.scale2 * (cr / sa) - lse_a + lse_b);
+    // cr = sum_c w(c) (O_T - O_S)[c] with w the teacher's (or, reversed, the student's) weights
+    const float kl = p.reverse ? kLn2 * (-p.scale2 * (cr / sb) - lse_b + lse_a)
+                               : kLn2 * (p.scale2 * (cr / sa) - lse_a + lse_b);
     p.kl[t] = on ? (kl < 0.f ? 0.f : kl) : 0.f;  // rounding may dip below 0; NaN stays NaN
     if (p.nll_s != nullptr) p.nll_s[t] = nll_s;
     if (p.nll_t != nullptr) p.nll_t[t] = nll_t;
@@ -422,7 +425,10 @@ __global__ void __launch_bounds__(256) select_kernel(
       }
     }
     const float dl = __fsub_rn(it, is);
-    bool k = (dl >= lo) && (dl <= hi);  // false for NaN
+    // what the interval tests (the filter ablation also tests the two IFDs alone) and whether
+    // its ends belong to it; every comparison is false for NaN
+    const float sc = (flags & 2) ? it : ((flags & 4) ? is : dl);
+    bool k = ((flags & 8) ? (sc > lo) : (sc >= lo)) && ((flags & 16) ? (sc < hi) : (sc <= hi));
     if (flags & 1) k = k && (it <= 1.0f);
     if (ifd_t != nullptr) ifd_t[i] = it;
     if (ifd_s != nullptr) ifd_s[i] = is;

@@ -349,6 +349,47 @@ def test_select_matches_float32_oracle_bit_for_bit():
         assert np.array_equal(keep.cpu().numpy(), o[3]) and int(n.item()) == o[4]
 
 
+def test_filter_ablation_scopes_match_float32_oracle_bit_for_bit():
+    rng = np.random.default_rng(1)
+    S, N = 1001, 700
+    count = rng.integers(0, 30, size=S).astype(np.int32)
+    s_sum = (rng.random(S) * 20).astype(np.float32)
+    t_sum = (rng.random(S) * 20).astype(np.float32)
+    cond = rng.integers(0, S, size=N).astype(np.int32)
+    unc = rng.integers(0, S, size=N).astype(np.int32)
+    # make some scores land exactly on the ends 0 and 1
+    s_sum[cond[:40]] = 0.0
+    t_sum[cond[40:80]] = t_sum[unc[40:80]] * count[cond[40:80]] / np.maximum(count[unc[40:80]], 1)
+    to = lambda x: torch.from_numpy(x).to(DEV)
+    inf = float("inf")
+    cases = [(B.NPD_SELECT_SCORE_IFD_TEACHER, 0.0, 1.0, dict(score="ifd_teacher")),
+             (B.NPD_SELECT_SCORE_IFD_STUDENT, 0.0, 1.0, dict(score="ifd_student")),
+             (B.NPD_SELECT_LO_EXCLUSIVE, 0.0, inf, dict(lo_inclusive=False)),
+             (B.NPD_SELECT_HI_EXCLUSIVE, -inf, 1.0, dict(hi_inclusive=False)),
+             (B.NPD_SELECT_SCORE_IFD_STUDENT | B.NPD_SELECT_LO_EXCLUSIVE | B.NPD_SELECT_HI_EXCLUSIVE, 0.0, 1.0,
+              dict(score="ifd_student", lo_inclusive=False, hi_inclusive=False))]
+    for flags, lo, hi, kw in cases:
+        keep, n = B.npd_select(to(cond), to(unc), to(s_sum), to(t_sum), to(count), lo, hi, flags)[3:]
+        o = orc.delta_ifd_select(cond, unc, s_sum, t_sum, count, lo, hi, dtype=np.float32, **kw)
+        assert np.array_equal(keep.cpu().numpy(), o[3]) and int(n.item()) == o[4], kw
+    assert B.lib().npd_select(N, 1, 1, 1, 1, 1, S, C.c_float(0), C.c_float(1), 6, 0, 0, 0, 1, 1, None) == B.NPD_EINVAL
+
+
+@pytest.mark.parametrize("tau", [1.0, 2.0])
+def test_policy_lag_monitor_reverse_kl(tau):
+    b = syn.scaled("c2", device=DEV, T=700, d=128, V=3000, min_len=20, max_len=300)
+    b.tau = tau
+    step = run_step(b, grads=False, flags=B.NPD_KD_REVERSE_KL)
+    H, W, Z, y, m = oracle_inputs(b)
+    assert_losses_close(host(step.kl), orc.reverse_kl_token(H, W, Z, m, tau), "reverse kl")
+    _, ns, nt = orc.kd_token_losses(H, W, Z, y, m, tau)
+    assert_losses_close(host(step.nll_student), ns, "nll_student")
+    assert_losses_close(host(step.nll_teacher), nt, "nll_teacher")
+    a = B.npd_kd_args.from_buffer_copy(run_step(b).args)
+    a.flags = B.NPD_KD_REVERSE_KL            # with gradients requested: refused
+    assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EINVAL
+
+
 def test_host_buffer_entry_point_matches_device_entry_point():
     b = syn.scaled("c2", device=DEV, T=300, d=64, V=520, min_len=20, max_len=90)
     ref = run_step(b)
