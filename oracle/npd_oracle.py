@@ -65,6 +65,7 @@ __all__ = [
     "ifd_scores",
     "delta_ifd_select",
     "nearest_rank_percentile",
+    "pack_first_fit_decreasing",
 ]
 
 
@@ -435,3 +436,45 @@ def nearest_rank_percentile(values, q: float) -> float:
         return float("nan")
     k = int(np.ceil(q * v.size)) - 1
     return float(v[min(max(k, 0), v.size - 1)])
+
+
+# --------------------------------------------------------------------------- #
+# Sequence packing (Algorithm 1, Phase 1: S_pack <- Pack(D_select, Length = L))
+# --------------------------------------------------------------------------- #
+
+def pack_first_fit_decreasing(lengths, keep, capacity: int):
+    """Packs the kept samples into rows of at most ``capacity`` tokens.
+
+    The paper names the step but not the algorithm; the reading taken is first-fit
+    decreasing: the kept samples are visited from the longest to the shortest (ties: lower
+    sample index first) and each goes into the first row, in order of creation, that still
+    has room; if none has, a new row is opened.  A sample longer than the capacity is cut to
+    the capacity (a row is a fixed-length sequence).  Samples of length 0 are dropped.
+
+    Returns (order, row_of, cu_seqlens, row_ptr):
+      order[j]      sample placed j-th in the packed stream (rows back to back, samples
+                    within a row in the order they were placed),
+      row_of[j]     its row,
+      cu_seqlens    [len(order)+1] token boundaries of the packed stream,
+      row_ptr       [rows+1] index into ``order`` where each row starts.
+    """
+    lengths = np.asarray(lengths, dtype=np.int64)
+    keep = np.ones(lengths.size, dtype=bool) if keep is None else np.asarray(keep).astype(bool)
+    cand = [i for i in range(lengths.size) if keep[i] and lengths[i] > 0]
+    cand.sort(key=lambda i: (-min(int(lengths[i]), capacity), i))
+    rows, room = [], []
+    for i in cand:
+        n = min(int(lengths[i]), capacity)
+        for r in range(len(rows)):
+            if room[r] >= n:
+                rows[r].append(i)
+                room[r] -= n
+                break
+        else:
+            rows.append([i])
+            room.append(capacity - n)
+    order = [i for r in rows for i in r]
+    row_of = [r for r, members in enumerate(rows) for _ in members]
+    cu = np.concatenate([[0], np.cumsum([min(int(lengths[i]), capacity) for i in order])]).astype(np.int32)
+    row_ptr = np.concatenate([[0], np.cumsum([len(m) for m in rows])]).astype(np.int32)
+    return (np.asarray(order, dtype=np.int32), np.asarray(row_of, dtype=np.int32), cu, row_ptr)

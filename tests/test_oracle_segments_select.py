@@ -218,3 +218,56 @@ def test_reverse_kl_is_the_forward_kl_with_the_roles_swapped():
     from scipy.special import rel_entr, softmax
     ref = rel_entr(softmax(H @ W.T, axis=1), softmax(G, axis=1)).sum(axis=1) * m
     assert np.allclose(orc.reverse_kl_token(H, W, G, m), ref, atol=1e-13)
+
+
+# ----------------------------------------------------------------------------------------------
+# Pack(D_select, Length = L): first-fit decreasing
+# ----------------------------------------------------------------------------------------------
+def _min_rows_brute_force(sizes, cap):
+    """Smallest number of rows of capacity cap that hold all sizes (tiny inputs only)."""
+    best = [len(sizes)]
+    def place(k, room):
+        if len(room) >= best[0]:
+            return
+        if k == len(sizes):
+            best[0] = len(room)
+            return
+        for r in range(len(room)):
+            if room[r] >= sizes[k]:
+                room[r] -= sizes[k]
+                place(k + 1, room)
+                room[r] += sizes[k]
+        room.append(cap - sizes[k])
+        place(k + 1, room)
+        room.pop()
+    place(0, [])
+    return best[0]
+
+
+def test_packing_worked_example():
+    # lengths 5 4 3 3 2 into rows of 8, all kept: 5 opens row 0, 4 opens row 1, the first 3 joins
+    # row 0 (5+3), the second 3 joins row 1 (4+3), 2 fits nowhere (rooms 0 and 1) -> row 2
+    order, row_of, cu, ptr = orc.pack_first_fit_decreasing([3, 5, 2, 4, 3], None, 8)
+    assert order.tolist() == [1, 0, 3, 4, 2] and row_of.tolist() == [0, 0, 1, 1, 2]
+    assert cu.tolist() == [0, 5, 8, 12, 15, 17] and ptr.tolist() == [0, 2, 4, 5]
+
+
+def test_packing_invariants_and_quality():
+    rng = np.random.default_rng(3)
+    for trial in range(30):
+        n = int(rng.integers(1, 9))
+        cap = int(rng.integers(4, 12))
+        lengths = rng.integers(0, cap + 3, size=n)
+        keep = rng.random(n) < 0.8
+        order, row_of, cu, ptr = orc.pack_first_fit_decreasing(lengths, keep, cap)
+        want = sorted(i for i in range(n) if keep[i] and lengths[i] > 0)
+        assert sorted(order.tolist()) == want                       # every kept sample exactly once
+        sizes = np.minimum(lengths[order], cap)
+        assert np.array_equal(np.diff(cu), sizes)
+        for r in range(len(ptr) - 1):
+            assert sizes[ptr[r]:ptr[r + 1]].sum() <= cap             # no row overflows
+            assert np.all(row_of[ptr[r]:ptr[r + 1]] == r)
+        if want:
+            opt = _min_rows_brute_force(sorted(np.minimum(lengths[want], cap).tolist(), reverse=True), cap)
+            rows = len(ptr) - 1
+            assert opt <= rows <= (11 * opt + 6) // 9 + 1            # the known first-fit-decreasing bound
