@@ -223,6 +223,25 @@ int npd_select(int32_t N, const int32_t* cond_seg, const int32_t* uncond_seg,
                float* ifd_teacher, float* ifd_student, float* delta,
                uint8_t* keep, int32_t* n_keep, void* cuda_stream);
 
+/*
+ * HOST (all pointers are HOST pointers; no GPU work).  Sequence packing of Algorithm 1,
+ * Phase 1: S_pack <- Pack(D_select, Length = capacity).  The paper names the step, not the
+ * algorithm; this is first-fit decreasing: kept samples (keep[i] != 0, or all if keep is NULL)
+ * with length > 0 are visited from the longest to the shortest (ties: lower index first) and
+ * put into the first row, in order of creation, with enough room, else into a new row.  A
+ * sample longer than `capacity` is cut to `capacity`.
+ *   order[j]      sample placed j-th in the packed stream (rows back to back)      [<= N]
+ *   row_of[j]     its row                                                          [<= N]
+ *   cu_seqlens    token boundaries of the packed stream, ready for npd_kd_args     [<= N+1]
+ *   row_ptr       index into order where each row starts, row_ptr[rows] = placed   [<= N+1]
+ *   n_placed, n_rows   how many samples were placed and how many rows were opened
+ * Output arrays must hold N (resp. N+1) entries.  NPD_EINVAL on NULL outputs, N < 0 or
+ * capacity < 1.  Cost O(N log N + N * rows).
+ */
+int npd_pack_sequences(int32_t N, const int32_t* lengths, const uint8_t* keep, int32_t capacity,
+                       int32_t* order, int32_t* row_of, int32_t* cu_seqlens, int32_t* row_ptr,
+                       int32_t* n_placed, int32_t* n_rows);
+
 /* Synchronises `cuda_stream`, then reads the device-side status word of a
  * workspace that npd_kd_fwd_bwd used into *host_status (HOST): NPD_OK,
  * NPD_ESEQ or NPD_ETIMEOUT.  Returns NPD_ECUDA if the stream itself failed. */

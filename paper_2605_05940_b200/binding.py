@@ -30,7 +30,7 @@ NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32 =
 
 EXPORTS = ("npd_workspace_bytes", "npd_phase_count", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
            "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16",
-           "npd_kd_forward_noalloc")
+           "npd_kd_forward_noalloc", "npd_pack_sequences")
 NPD_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 
@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
         l.npd_last_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
         l.npd_last_launch_count.argtypes = []
         l.npd_kd_forward_noalloc.argtypes = [C.POINTER(npd_kd_args), C.c_void_p, C.POINTER(C.c_int32)]
+        l.npd_pack_sequences.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_int32] + [C.c_void_p] * 6
         l.npd_gemm_bf16.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int32,
                                     C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64,
                                     C.c_int32, C.c_int32, C.c_void_p]
@@ -172,7 +173,7 @@ def npd_kd_forward_noalloc(args: npd_kd_args, stream=None, want_status: bool = F
     With want_status the call synchronises the stream and returns the device status."""
     st = C.c_int32(0)
     _check(lib().npd_kd_forward_noalloc(C.byref(args), _stream(stream), C.byref(st) if want_status else None),
-           "npd_kd_forward_noalloc")
+           "npd_kd_forward_noalloc", "npd_pack_sequences")
     return st.value if want_status else None
 
 
@@ -221,6 +222,23 @@ def npd_select(cond_seg, uncond_seg, nll_s_sum, nll_t_sum, count, lo: float, hi:
                             _ptr(count), S, float(lo), float(hi), int(flags), _ptr(ifd_t), _ptr(ifd_s),
                             _ptr(delta), _ptr(keep), _ptr(n_keep), _stream(stream)), "npd_select")
     return ifd_t, ifd_s, delta, keep, n_keep
+
+
+def npd_pack_sequences(lengths, keep, capacity: int):
+    """First-fit-decreasing packing of the kept samples into rows of `capacity` tokens (host only).
+    lengths: int32 array-like, keep: uint8 array-like or None.  Returns numpy arrays
+    (order, row_of, cu_seqlens, row_ptr)."""
+    import numpy as np
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    N = lengths.size
+    k = None if keep is None else np.ascontiguousarray(keep, dtype=np.uint8)
+    order, row_of = np.empty(N, np.int32), np.empty(N, np.int32)
+    cu, ptr = np.empty(N + 1, np.int32), np.empty(N + 1, np.int32)
+    placed, rows = C.c_int32(0), C.c_int32(0)
+    _check(lib().npd_pack_sequences(N, lengths.ctypes.data, None if k is None else k.ctypes.data, int(capacity),
+                                    order.ctypes.data, row_of.ctypes.data, cu.ctypes.data, ptr.ctypes.data,
+                                    C.addressof(placed), C.addressof(rows)), "npd_pack_sequences")
+    return order[:placed.value], row_of[:placed.value], cu[:placed.value + 1], ptr[:rows.value + 1]
 
 
 def npd_gemm_bf16(A, B, out, *, a_mn_major=False, b_mn_major=False, out_mode=NPD_GEMM_STORE_F32,

@@ -12,6 +12,7 @@
 #include <cstdint>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "gemm_sm100.cuh"
 #include "kd_tile_sm100.cuh"
@@ -640,6 +641,48 @@ int npd_select(int32_t N, const int32_t* cond_seg, const int32_t* uncond_seg, co
                                                  lo, hi, flags, ifd_teacher, ifd_student, delta, keep,
                                                  n_keep);
   return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
+}
+
+int npd_pack_sequences(int32_t N, const int32_t* lengths, const uint8_t* keep, int32_t capacity,
+                       int32_t* order, int32_t* row_of, int32_t* cu_seqlens, int32_t* row_ptr,
+                       int32_t* n_placed, int32_t* n_rows) {
+  if (N < 0 || capacity < 1 || (N > 0 && lengths == nullptr) || order == nullptr || row_of == nullptr ||
+      cu_seqlens == nullptr || row_ptr == nullptr || n_placed == nullptr || n_rows == nullptr)
+    return NPD_EINVAL;
+  std::vector<int32_t> cand;
+  cand.reserve(N);
+  for (int32_t i = 0; i < N; ++i)
+    if ((keep == nullptr || keep[i] != 0) && lengths[i] > 0) cand.push_back(i);
+  auto len = [&](int32_t i) { return std::min(lengths[i], capacity); };
+  std::stable_sort(cand.begin(), cand.end(), [&](int32_t a, int32_t b) { return len(a) > len(b); });
+  std::vector<int32_t> room;                       // free tokens of every open row
+  std::vector<std::vector<int32_t>> members;       // samples of every row, in placing order
+  for (int32_t i : cand) {
+    const int32_t n = len(i);
+    size_t r = 0;
+    while (r < room.size() && room[r] < n) ++r;    // first row with room
+    if (r == room.size()) {
+      room.push_back(capacity);
+      members.emplace_back();
+    }
+    room[r] -= n;
+    members[r].push_back(i);
+  }
+  int32_t j = 0;
+  cu_seqlens[0] = 0;
+  for (size_t r = 0; r < members.size(); ++r) {
+    row_ptr[r] = j;
+    for (int32_t i : members[r]) {
+      order[j] = i;
+      row_of[j] = static_cast<int32_t>(r);
+      cu_seqlens[j + 1] = cu_seqlens[j] + len(i);
+      ++j;
+    }
+  }
+  row_ptr[members.size()] = j;
+  *n_placed = j;
+  *n_rows = static_cast<int32_t>(members.size());
+  return NPD_OK;
 }
 
 int npd_last_status(const void* workspace, void* cuda_stream, int32_t* host_status) {

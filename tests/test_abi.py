@@ -128,3 +128,18 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/libnpd.so")
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         B.lib()
+
+
+def test_sequence_packer_matches_the_oracle():
+    # host-only entry point: runs without a GPU
+    import numpy as np
+    from oracle import npd_oracle as orc
+    rng = np.random.default_rng(0)
+    for n, cap in [(0, 8), (1, 8), (5, 8), (200, 512), (3000, 32768)]:
+        lengths = rng.integers(0, cap + cap // 4 + 2, size=n).astype(np.int32)
+        for keep in (None, (rng.random(n) < 0.7).astype(np.uint8)):
+            got = B.npd_pack_sequences(lengths, keep, cap)
+            want = orc.pack_first_fit_decreasing(lengths, keep, cap)
+            for g, w in zip(got, want):
+                assert np.array_equal(g, w)
+    assert B.lib().npd_pack_sequences(3, None, None, 8, None, None, None, None, None, None) == B.NPD_EINVAL
