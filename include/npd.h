@@ -285,7 +285,7 @@ int npd_last_launch_count(void);
  * stores the device-side status (NPD_OK, NPD_ESEQ, NPD_ETIMEOUT) there, as
  * npd_last_status would; if NULL the call only enqueues.
  */
-#define NPD_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
+#define NPD_STATIC_SCRATCH_BYTES (48u * 1024u * 1024u)
 int npd_kd_forward_noalloc(const npd_kd_args* args, void* cuda_stream, int32_t* host_status);
 
 /* out_mode of npd_gemm_bf16 */

@@ -31,7 +31,7 @@ NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32 =
 EXPORTS = ("npd_workspace_bytes", "npd_phase_count", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
            "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16",
            "npd_kd_forward_noalloc", "npd_pack_sequences")
-NPD_STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
+NPD_STATIC_SCRATCH_BYTES = 48 * 1024 * 1024
 
 
 class NpdError(RuntimeError):
@@ -173,7 +173,7 @@ def npd_kd_forward_noalloc(args: npd_kd_args, stream=None, want_status: bool = F
     With want_status the call synchronises the stream and returns the device status."""
     st = C.c_int32(0)
     _check(lib().npd_kd_forward_noalloc(C.byref(args), _stream(stream), C.byref(st) if want_status else None),
-           "npd_kd_forward_noalloc", "npd_pack_sequences")
+           "npd_kd_forward_noalloc")
     return st.value if want_status else None
 
 

@@ -39,19 +39,16 @@ struct GemmProblem {
   int k_splits;    // > 1 only with out_reduce
   int out_f32;     // output elements: 1 = fp32, 0 = bf16
   int out_reduce;  // 1 = D += acc (atomic, any number of adders), 0 = D = acc
-  // Row-block indirection for the backward over the 128-row blocks of a packed batch that hold
-  // loss tokens (blocks[i] = first row of block i, nblocks[0] = how many; both on the device):
-  int dyn_m;       // M = 128 * nblocks[0]: A's rows are the listed blocks, stored back to back
-  int dyn_k;       // K = 128 * nblocks[0]: A's k-extent likewise
-  int map_bk;      // B's k coordinate of compact k-row i*128+j is blocks[i]+j
-  int map_om;      // output row of compact row i*128+j is blocks[i]+j
+  // Extents only known on the device (the backward runs over the compact rows of a packed
+  // batch, nblocks[0] blocks of 128):
+  int dyn_m;       // M = 128 * nblocks[0]
+  int dyn_k;       // K = 128 * nblocks[0]
 };
 
 struct GemmParams {
   GemmProblem pr[2];
   int nprob;           // 1 or 2
   const int* nblocks;  // device; read only when a problem has dyn_m / dyn_k
-  const int* blocks;   // device; read only when a problem has map_bk / map_om
   int* status;         // device status word
 };
 
@@ -231,8 +228,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
           const uint32_t fb = full_leader + 8 * s;
           const uint32_t sa = smem_u32(smem_a + s * A_BYTES), sb = smem_u32(smem_b + s * B_BYTES);
           const int k0 = kt * BK;
-          // B's k rows: straight, or the rows of the kt/2-th listed block
-          const int kb = g.map_bk ? __ldg(p.blocks + (kt >> 1)) + (kt & 1) * BK : k0;
+          const int kb = k0;
           if (g.a_mn) {
 #pragma unroll
             for (int j = 0; j < BM / 64; ++j) tma_load_2d_pair(sa + j * 8192, ta, fb, m0 + 64 * j, k0);
@@ -314,8 +310,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
       const CUtensorMap* to = prob ? &tmap_o1 : &tmap_o0;
       const int m0 = u.m0 + static_cast<int>(rank) * BM;
       const bool rows_inside = m0 < g.M;          // else this CTA's 128 rows lie beyond M: nothing to store
-      // output rows: straight, or the rows of the listed block
-      const int out_row0 = (g.map_om && rows_inside) ? __ldg(p.blocks + (m0 >> 7)) : m0;
+      const int out_row0 = m0;
       const bool no_k = u.kt0 == u.kt1;           // empty k range: the accumulators hold nothing, D = 0
       const int gcols = (BNS / 2) * u.ns;         // accumulator columns this group drains
       const int c0 = grp * gcols;                 // the first of them

@@ -52,9 +52,10 @@ enum : int { kPMaxA = 0, kPSumA, kPCross, kPMaxB, kPSumB, kPSumA1, kPSumB1, kPFi
 struct KdTileParams {
   int T, V;
   int ksteps;       // d / 64
-  const int* plan;  // {128-row blocks that hold loss tokens, pairs of them, forward runs, 0} (device)
-  const int* list;  // first packed row of every such block, in order; a pair of CTAs owns two
-                    // consecutive entries
+  // The kernels work on the COMPACT rows: the tokens that carry loss, in packed order, numbered
+  // 0..Tc-1 and cut into blocks of 128; a pair of CTAs owns two consecutive blocks.
+  const int* plan;  // {blocks, pairs of blocks, forward runs, Tc}, written on the device
+  const int* rows;  // [blocks*128] packed row (token) of every compact row; 0 beyond Tc
   int group_pairs;  // pairs of blocks per group: units are ordered group by group (within a group:
                     // pair fastest, then run), so that the H rows the CTA pairs work on at
                     // any one time stay in L2 while the W tiles are shared by a whole group
@@ -68,19 +69,20 @@ struct KdTileParams {
   int reverse;      // 1: the cross term is weighted by the student's probabilities (the divergence
                     // of the policy-lag monitor, student || given logits) instead of the teacher's
   // gradient
+  // per-token arrays below are indexed by COMPACT row
   const float* lse2_a;  // [T] log2-sum-exp2 of the scaled teacher logits
   const float* lse2_b;  // [T] same for the student
   const float* coef;    // [T] grad_scale * m_t * lambda / tau
   // composite objective only (Eq. 1)
   const float* coef_ce;   // [T] grad_scale * m_t * [y_t >= 0] * (1 - lambda)
   const float* lse2_b1;   // [T] log2-sum-exp2 of the student logits * log2(e) (temperature 1)
-  const int32_t* labels;  // [T]
+  const int32_t* labels;  // [T], by token
   // top-k teacher only (kSparse)
-  const int32_t* tk_idx;  // [T, topk] vocabulary indices of the stored teacher logits
-  const float* tk_cp;     // [T, topk] coef_t * p_T(j): what the gradient subtracts at column idx[t,j]
+  const int32_t* tk_idx;  // [T, topk] vocabulary indices of the stored teacher logits, by token
+  const float* tk_cp;     // [T, topk] coef_t * p_T(j): what the gradient subtracts at column idx[t,j],
+                          // by compact row
   int topk;               // <= kMaxTopK
-  int g_col0;           // vocabulary column that scratch column 0 holds; scratch row = position in
-                        // the block list * 128 + row within the block
+  int g_col0;           // vocabulary column that scratch column 0 holds; scratch row = compact row
   int* status;
 };
 
@@ -166,16 +168,15 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   const int nact = p.plan[0], pairs = p.plan[1];
   const int nsplit = kMode == kForward ? p.plan[2] : p.vt_count;
   const int units = pairs * nsplit;
-  // slot = this CTA's position in the block list, r = that block's first packed row, or -1
-  // when the list has an odd length and this CTA has no block (it then stages the rows from 0
-  // and writes nothing).
+  // slot = this CTA's block of compact rows, r = its first compact row, or -1 when the number of
+  // blocks is odd and this CTA has none (it then stages block 0 and writes nothing).
   const int per_group = p.group_pairs * nsplit;  // units of a full group
   auto run_of = [&](int u, int& slot, int& r, int& s, int& vt0, int& vt1) {
     const int gi = u / per_group, local = u - gi * per_group;
     const int gsize = min(p.group_pairs, pairs - gi * p.group_pairs);
     s = local / gsize;
     slot = 2 * (gi * p.group_pairs + local % gsize) + static_cast<int>(rank);
-    r = slot < nact ? __ldg(p.list + slot) : -1;
+    r = slot < nact ? slot * BM : -1;
     vt0 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * s / nsplit);
     vt1 = p.vt_begin + static_cast<int>(static_cast<long long>(p.vt_count) * (s + 1) / nsplit);
   };
@@ -245,23 +246,30 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     }
   } else if (warp == 2) {
     // ---------------------- teacher producer ----------------------
-    if (!kSparse && lane == 0) {
+    // The teacher rows of a block are scattered over the packed batch (the masked tokens in
+    // between are left out), so a 128 x 64 sub-tile is fetched as 32 four-row gathers, one per
+    // lane: lane l brings the block's rows 4l..4l+3 to their place in the swizzled sub-tile.
+    if (!kSparse) {
       uint32_t zit = 0;  // sub-tile pairs issued; both halves advance together
       bool ok = true;
       for (int u = cluster_id; u < units && ok; u += num_clusters) {
         int slot, r, s, vt0, vt1;
         run_of(u, slot, r, s, vt0, vt1);
-        const int rl = r < 0 ? 0 : r;
+        int tr[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) tr[i] = r < 0 ? 0 : __ldg(p.rows + r + 4 * lane + i);
         for (int vt = vt0; vt < vt1 && ok; ++vt) {
           for (int j = 0; j < BN / 2 / ZSUB_COLS && ok; ++j, ++zit) {
             const uint32_t q = zit % ZQ, ph = (zit / ZQ) & 1;
             for (int half = 0; half < 2; ++half) {
               const int col = vt * BN + half * (BN / 2) + j * ZSUB_COLS;
               const uint32_t bi = 8 * (half * ZQ + q);
-              if (!(ok = mbar_wait(zempty0 + bi, ph ^ 1, abort_flag))) break;
-              mbar_arrive_expect_tx(zfull0 + bi, ZSUB_BYTES);
-              tma_load_2d(smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES), &tmap_t, zfull0 + bi,
-                          col, rl);
+              ok = __all_sync(0xffffffffu, mbar_wait(zempty0 + bi, ph ^ 1, abort_flag));
+              if (!ok) break;
+              if (lane == 0) mbar_arrive_expect_tx(zfull0 + bi, ZSUB_BYTES);
+              __syncwarp();
+              tma_gather4_2d(smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES) + lane * 512, &tmap_t,
+                             zfull0 + bi, col, tr[0], tr[1], tr[2], tr[3]);
             }
           }
         }
@@ -285,21 +293,22 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     for (int u = cluster_id; u < units && ok; u += num_clusters) {
       int slot, r, s, vt0, vt1;
       run_of(u, slot, r, s, vt0, vt1);
-      const int row = r < 0 ? p.T : r + row_local;  // token row; >= T: nothing to read or write
+      const int tc = p.plan[3];
+      const int row = r < 0 ? tc : r + row_local;  // compact row; >= Tc: nothing to read or write
       // forward state (base-2 domain): running max / sum of the scaled teacher (a) and student (b)
       float m_a = -INFINITY, s_a = 0.f, cross = 0.f, m_b = -INFINITY, s_b = 0.f, s_a1 = 0.f, s_b1 = 0.f;
       // rows without a token (beyond T, or a CTA without a block): probabilities 0, gradient 0
       float g_lse_a = 1e30f, g_lse_b = 1e30f, g_coef = 0.f;
       float g_cce = 0.f, g_lse_b1 = 1e30f;  // cross-entropy term of the composite objective
       int g_y = -1;
-      if (kMode == kGradient && row < p.T) {
+      if (kMode == kGradient && row < tc) {
         g_lse_a = p.lse2_a[row];
         g_lse_b = p.lse2_b[row];
         g_coef = p.coef[row];
         if (kComposite) {
           g_cce = p.coef_ce[row];
           g_lse_b1 = p.lse2_b1[row];
-          g_y = g_cce != 0.f ? p.labels[row] : -1;
+          g_y = g_cce != 0.f ? p.labels[__ldg(p.rows + row)] : -1;
         }
       }
       // top-k teacher: this row's stored columns and what to subtract there
@@ -308,8 +317,8 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       if (kSparse && kMode == kGradient) {
 #pragma unroll
         for (int j = 0; j < kMaxTopK; ++j) {
-          const bool have = row < p.T && j < p.topk;
-          tki[j] = have ? p.tk_idx[static_cast<size_t>(row) * p.topk + j] : -1;
+          const bool have = row < tc && j < p.topk;
+          tki[j] = have ? p.tk_idx[static_cast<size_t>(__ldg(p.rows + row)) * p.topk + j] : -1;
           tkc[j] = have ? p.tk_cp[static_cast<size_t>(row) * p.topk + j] : 0.f;
         }
       }
@@ -468,7 +477,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             if (lg == 0 && lane == 0) {
               if (r >= 0) {
                 tma_store_2d(&tmap_g, smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES),
-                             sub_col0 - p.g_col0, slot * BM);
+                             sub_col0 - p.g_col0, r);
                 tma_store_commit();
                 tma_store_wait_read<0>();
               }
@@ -485,7 +494,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(tempty_leader + 8 * buf);
       }
-      if (kMode == kForward && ok && row < p.T) {
+      if (kMode == kForward && ok && row < tc) {
         float* dst = p.partials + (static_cast<size_t>(2 * s + half) * kPFields) * p.T + row;
         dst[static_cast<size_t>(kPMaxA) * p.T] = m_a;
         dst[static_cast<size_t>(kPSumA) * p.T] = s_a;

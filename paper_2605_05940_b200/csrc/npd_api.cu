@@ -74,9 +74,8 @@ struct Plan {
   int chunk_cols;     // vocabulary columns per gradient chunk (multiple of 256)
   int nchunks;
   int dh_ksplits;     // split-K of the dH product of a full chunk
-  bool dh_direct;     // dH stored straight to the output (one chunk, no split-K); else fp32 atomics
   bool grads;
-  size_t off_status, off_plan, off_list, off_partials, off_lse_a, off_lse_b, off_coef, off_coef_ce,
+  size_t off_status, off_plan, off_rows, off_cidx, off_hc, off_partials, off_lse_a, off_lse_b, off_coef, off_coef_ce,
       off_lse_b1, off_tkcp, off_g, off_dh, total;
 };
 
@@ -110,14 +109,18 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   const long long tiles_h = static_cast<long long>((pl->row_blocks + 1) / 2) * ((a->d + 511) / 512);
   const int want = static_cast<int>((8ll * pl->clusters + tiles_h - 1) / tiles_h);
   pl->dh_ksplits = std::max(1, std::min(want, ksteps_h / 48));
-  pl->dh_direct = pl->nchunks == 1 && pl->dh_ksplits == 1;
   size_t off = 0;
   pl->off_status = off;
   off += 1024;
   pl->off_plan = off;
   off += 1024;
-  pl->off_list = off;
-  off = align_up(off + sizeof(int) * static_cast<size_t>(pl->row_blocks), 1024);
+  const size_t crows = static_cast<size_t>(pl->row_blocks) * 128;  // upper bound of the compact rows
+  pl->off_rows = off;
+  off = align_up(off + sizeof(int) * crows, 1024);
+  pl->off_cidx = off;
+  off = align_up(off + sizeof(int) * static_cast<size_t>(a->T), 1024);
+  pl->off_hc = off;  // hidden states of the compact rows, bf16 [crows, d]
+  off = align_up(off + 2 * crows * a->d, 1024);
   pl->off_partials = off;
   off = align_up(off + sizeof(float) * 2 * pl->nsplit_max * kPFields * static_cast<size_t>(a->T), 1024);
   pl->off_lse_a = off;
@@ -138,9 +141,9 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   pl->off_g = off;
   pl->off_dh = off;
   if (pl->grads) {
-    off = align_up(off + 2 * static_cast<size_t>(pl->row_blocks) * 128 * cc, 1024);
-    pl->off_dh = off;
-    if (!pl->dh_direct) off = align_up(off + sizeof(float) * static_cast<size_t>(a->T) * a->d, 1024);
+    off = align_up(off + 2 * crows * cc, 1024);
+    pl->off_dh = off;  // fp32 dH accumulator over the compact rows
+    off = align_up(off + sizeof(float) * crows * a->d, 1024);
   }
   pl->total = off;
   return NPD_OK;
@@ -204,14 +207,12 @@ struct GemmOperands {
   long long ldb;
   void* out;
   long long ldo;
-  long long b_rows;    // rows of B's / the output's memory when they are addressed through the
-  long long out_rows;  // block list (else unused)
 };
 
 // One launch for one or two problems (see gemm_sm100.cuh for how the units are dealt).
-// a_rows / a_kext: extents of A's tensor map when M or K is only known on the device.
+// An extent only known on the device (dyn_m / dyn_k) is 128 * max_blocks as far as the maps go.
 int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const int* nblocks,
-                const int* blocks, int max_blocks, int* status, int sms, cudaStream_t st) {
+                int max_blocks, int* status, int sms, cudaStream_t st) {
   using namespace gemm_cfg;
   CUtensorMap maps[6];
   GemmParams gp{};
@@ -221,8 +222,7 @@ int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const
     const GemmProblem& g = pr[j];
     // extents as the maps see them: device-side dimensions take their upper bound
     const uint64_t am = g.dyn_m ? 128ull * max_blocks : g.M, ak = g.dyn_k ? 128ull * max_blocks : g.K;
-    const uint64_t bk = (g.dyn_k || g.map_bk) ? static_cast<uint64_t>(ops[j].b_rows) : g.K;
-    const uint64_t om = (g.dyn_m || g.map_om) ? static_cast<uint64_t>(ops[j].out_rows) : g.M;
+    const uint64_t bk = ak, om = am;
     const bool oka = g.a_mn ? make_map(&maps[3 * i], ops[j].A, am, ak, ops[j].lda, 64, 64)
                             : make_map(&maps[3 * i], ops[j].A, ak, am, ops[j].lda, 64, BM);
     const bool okb = g.b_mn ? make_map(&maps[3 * i + 1], ops[j].B, g.N, bk, ops[j].ldb, 64, 64)
@@ -237,7 +237,6 @@ int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const
   }
   gp.nprob = nprob;
   gp.nblocks = nblocks;
-  gp.blocks = blocks;
   gp.status = status;
   const int pairs = static_cast<int>(std::max<long long>(1, std::min<long long>(units, std::max(sms / 2, 1))));
   if (set_smem(gemm_bf16_kernel, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
@@ -318,7 +317,10 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   uint8_t* ws = static_cast<uint8_t*>(a->workspace);
   int* status = reinterpret_cast<int*>(ws + pl.off_status);
   int* plan = reinterpret_cast<int*>(ws + pl.off_plan);
-  int* list = reinterpret_cast<int*>(ws + pl.off_list);
+  int* rows = reinterpret_cast<int*>(ws + pl.off_rows);
+  int* cidx = reinterpret_cast<int*>(ws + pl.off_cidx);
+  __nv_bfloat16* hc = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_hc);
+  const uint64_t crows = static_cast<uint64_t>(pl.row_blocks) * 128;
   float* partials = reinterpret_cast<float*>(ws + pl.off_partials);
   float* lse_a = reinterpret_cast<float*>(ws + pl.off_lse_a);
   float* lse_b = reinterpret_cast<float*>(ws + pl.off_lse_b);
@@ -335,12 +337,13 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   const bool sparse = a->topk > 0;  // teacher stored as its top-k logits per token
   float* tk_cp = reinterpret_cast<float*>(ws + pl.off_tkcp);
   CUtensorMap mh, mw, mt;
-  if (!make_map(&mh, a->hidden, a->d, a->T, a->ldh, 64, 128) ||
+  // H is read as its compact copy; the teacher by four-row gathers (box one row high)
+  if (!make_map(&mh, hc, a->d, crows, a->d, 64, 128) ||
       !make_map(&mw, a->weight, a->d, a->V, a->ldw, 64, 128))
     return NPD_ECUDA;
   if (sparse) {
     mt = mh;  // never used: no teacher tiles are streamed
-  } else if (!make_map(&mt, a->teacher, a->V, a->T, a->ldt, 64, 128)) {
+  } else if (!make_map(&mt, a->teacher, a->V, a->T, a->ldt, 64, 1)) {
     return NPD_ECUDA;
   }
 
@@ -352,17 +355,13 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     ++g_launches;
   }
 
-  // ---- cover the tokens with loss by 128-row blocks; everything below works on those only ----
-  {
-    const int words = (a->T + 31) / 32;
-    const int bitmap_words = words <= 48 * 1024 ? words : 0;  // up to 192 KB of shared memory
-    if (bitmap_words * 4 > 48 * 1024 &&
-        set_smem(plan_blocks_kernel, bitmap_words * 4) != NPD_OK)
-      return NPD_ECUDA;
-    plan_blocks_kernel<<<1, 1024, bitmap_words * 4, st>>>(a->T, a->loss_mask, bitmap_words, pl.vtiles,
-                                                          pl.nsplit_max, pl.clusters, plan, list);
-  }
-  ++g_launches;
+  // ---- number the tokens with loss (compact rows) and gather their hidden states; everything
+  // below works on the compact rows only ----
+  plan_rows_kernel<<<1, 1024, 0, st>>>(a->T, a->loss_mask, pl.vtiles, pl.nsplit_max, pl.clusters, plan, rows,
+                                       cidx);
+  gather_hidden_rows_kernel<<<2 * di.sms, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(a->hidden), a->ldh,
+                                                        a->d, plan, rows, hc);
+  g_launches += 2;
   if (cudaGetLastError() != cudaSuccess) return NPD_ECUDA;
 
   rec.mark();
@@ -372,7 +371,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   kp.V = a->V;
   kp.ksteps = a->d / 64;
   kp.plan = plan;
-  kp.list = list;
+  kp.rows = rows;
   // a group's H rows (256 x d bf16 per pair) should fill at most a quarter of a 128 MB L2
   kp.group_pairs = static_cast<int>(std::max<long long>(4, (32ll << 20) / (512ll * a->d)));
   kp.vt_begin = 0;
@@ -392,6 +391,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     tp.V = a->V;
     tp.topk = a->topk;
     tp.plan = plan;
+    tp.cidx = cidx;
     tp.partials = partials;
     tp.hidden = static_cast<const __nv_bfloat16*>(a->hidden);
     tp.weight = static_cast<const __nv_bfloat16*>(a->weight);
@@ -422,6 +422,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   cp.d = a->d;
   cp.V = a->V;
   cp.plan = plan;
+  cp.cidx = cidx;
   cp.partials = partials;
   cp.hidden = static_cast<const __nv_bfloat16*>(a->hidden);
   cp.weight = static_cast<const __nv_bfloat16*>(a->weight);
@@ -460,22 +461,14 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   __nv_bfloat16* gbuf = reinterpret_cast<__nv_bfloat16*>(ws + pl.off_g);
   float* dh_acc = reinterpret_cast<float*>(ws + pl.off_dh);
   const long long ldg = pl.chunk_cols;
-  // rows of blocks without loss are never written by the contractions: they start as zeros
-  if (pl.dh_direct) {
-    if (cudaMemset2DAsync(a->d_hidden, static_cast<size_t>(a->ldh) * 2, 0, static_cast<size_t>(a->d) * 2,
-                          a->T, st) != cudaSuccess)
-      return NPD_ECUDA;
-  } else if (cudaMemsetAsync(dh_acc, 0, sizeof(float) * static_cast<size_t>(a->T) * a->d, st) !=
-             cudaSuccess) {
-    return NPD_ECUDA;
-  }
+  if (cudaMemsetAsync(dh_acc, 0, sizeof(float) * crows * a->d, st) != cudaSuccess) return NPD_ECUDA;
   for (int c = 0; c < pl.nchunks; ++c) {
     const int col0 = c * pl.chunk_cols;
     const int cols = std::min(pl.chunk_cols, a->V - col0);  // columns of this chunk inside V
     if (cols <= 0) break;
     const int cols_pad = std::min(pl.chunk_cols, pl.vtiles * 256 - col0);
     CUtensorMap mg;
-    if (!make_map(&mg, gbuf, cols_pad, static_cast<uint64_t>(pl.row_blocks) * 128, ldg, 64, 128))
+    if (!make_map(&mg, gbuf, cols_pad, crows, ldg, 64, 128))
       return NPD_ECUDA;
     KdTileParams gp = kp;
     gp.vt_begin = col0 / 256;
@@ -496,14 +489,13 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
 
     GemmProblem pr[2] = {};
     GemmOperands ops[2] = {};
-    // The logit-gradient block holds the active row blocks back to back (scratch row = position
-    // in the list * 128 + row within the block); H and dH are addressed through the list.
-    // dW[col0 .. col0+cols) = G_chunk^T H       (M = vocabulary rows, N = d, K = active token rows)
+    // Everything here lives on the compact rows: the logit-gradient block, the gathered hidden
+    // states and the fp32 dH accumulator.
+    // dW[col0 .. col0+cols) = G_chunk^T Hc      (M = vocabulary rows, N = d, K = compact rows)
     pr[0].M = cols;
     pr[0].N = a->d;
     pr[0].K = 0;
     pr[0].dyn_k = 1;
-    pr[0].map_bk = 1;
     pr[0].a_mn = 1;
     pr[0].b_mn = 1;
     pr[0].k_splits = 1;
@@ -513,34 +505,27 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
                         ? static_cast<void*>(static_cast<float*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw)
                         : static_cast<void*>(static_cast<__nv_bfloat16*>(a->d_weight) +
                                              static_cast<size_t>(col0) * a->ldw);
-    ops[0] = {gbuf, ldg, a->hidden, a->ldh, dw_rows, a->ldw, a->T, 0};
-    // dH (+)= G_chunk W[col0 .. col0+cols)      (M = active token rows, N = d, K = the chunk's columns)
+    ops[0] = {gbuf, ldg, hc, a->d, dw_rows, a->ldw};
+    // dH += G_chunk W[col0 .. col0+cols)        (M = compact rows, N = d, K = the chunk's columns)
     pr[1].M = 0;
     pr[1].dyn_m = 1;
-    pr[1].map_om = 1;
     pr[1].N = a->d;
     pr[1].K = cols;
     pr[1].a_mn = 0;
     pr[1].b_mn = 1;
+    pr[1].k_splits = std::max(1, std::min(pl.dh_ksplits, (cols + 63) / 64));
+    pr[1].out_f32 = 1;
+    pr[1].out_reduce = 1;
     const __nv_bfloat16* w_rows = static_cast<const __nv_bfloat16*>(a->weight) + static_cast<size_t>(col0) * a->ldw;
-    if (pl.dh_direct) {
-      pr[1].k_splits = 1;
-      pr[1].out_f32 = 0;
-      pr[1].out_reduce = 0;
-      ops[1] = {gbuf, ldg, w_rows, a->ldw, a->d_hidden, a->ldh, 0, a->T};
-    } else {
-      pr[1].k_splits = std::max(1, std::min(pl.dh_ksplits, (cols + 63) / 64));
-      pr[1].out_f32 = 1;
-      pr[1].out_reduce = 1;
-      ops[1] = {gbuf, ldg, w_rows, a->ldw, dh_acc, a->d, 0, a->T};
-    }
-    if ((rc = launch_gemm(2, pr, ops, plan, list, pl.row_blocks, status, di.sms, st)) != NPD_OK) return rc;
+    ops[1] = {gbuf, ldg, w_rows, a->ldw, dh_acc, a->d};
+    if ((rc = launch_gemm(2, pr, ops, plan, pl.row_blocks, status, di.sms, st)) != NPD_OK) return rc;
     rec.mark();
   }
-  if (!pl.dh_direct) {
+  {
+    // compact fp32 rows -> bf16 rows of the tokens; tokens without loss get zeros
     const long long n = static_cast<long long>(a->T) * (a->d / 8);
-    f32_to_bf16_rows_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(
-        dh_acc, a->T, a->d, static_cast<__nv_bfloat16*>(a->d_hidden), a->ldh);
+    scatter_dhidden_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(
+        dh_acc, cidx, a->T, a->d, static_cast<__nv_bfloat16*>(a->d_hidden), a->ldh);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) return NPD_ECUDA;
     rec.mark();
@@ -560,7 +545,7 @@ int npd_phase_count(const npd_kd_args* args, int32_t* out_groups, int32_t* out_c
   if (pl.grads)
     for (int c = 0; c < pl.nchunks; ++c)
       if (args->V - c * pl.chunk_cols > 0) ++chunks;
-  *out_groups = 2 + 2 * chunks + ((pl.grads && !pl.dh_direct) ? 1 : 0);
+  *out_groups = 2 + 2 * chunks + (pl.grads ? 1 : 0);
   if (out_chunks != nullptr) *out_chunks = chunks;
   return NPD_OK;
 }
@@ -775,8 +760,8 @@ int npd_gemm_bf16(int32_t M, int32_t N, int32_t K, const void* A, int64_t lda, i
   pr.k_splits = k_splits;
   pr.out_f32 = f32;
   pr.out_reduce = out_mode == NPD_GEMM_ADD_F32 || out_mode == NPD_GEMM_ATOMIC_F32;
-  const GemmOperands ops{A, lda, B, ldb, out, ldo, 0, 0};
-  return launch_gemm(1, &pr, &ops, nullptr, nullptr, 0, nullptr, di.sms, static_cast<cudaStream_t>(cuda_stream));
+  const GemmOperands ops{A, lda, B, ldb, out, ldo};
+  return launch_gemm(1, &pr, &ops, nullptr, 0, nullptr, di.sms, static_cast<cudaStream_t>(cuda_stream));
 }
 
 }  // extern "C"

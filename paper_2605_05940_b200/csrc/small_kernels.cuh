@@ -42,64 +42,82 @@ __host__ __device__ inline int choose_nsplit(int pairs, int vtiles, int clusters
   return best;
 }
 
-// One CTA.  Covers the tokens that carry loss (m_t = 1) with 128-row blocks: a block starts at
-// the first such token that no earlier block covers and spans the 128 packed rows from there,
-// so the blocks are disjoint and skip the masked stretches (prompts) between them.  Rows outside
-// every block have zero loss and zero gradient, and no tile of any later kernel is spent on
-// them.  list[i] = first row of block i; plan = {blocks, pairs of blocks, forward runs, 0}.
-// Tokens are first marked in a bitmap in shared memory (bitmap_words 32-bit words, enough for
-// T bits); when T is too large for that the blocks fall back to the aligned grid 0, 128, 256...
-// with the blocks that hold no loss token left out.
-__global__ void __launch_bounds__(1024) plan_blocks_kernel(int T, const uint8_t* __restrict__ mask,
-                                                           int bitmap_words, int vtiles, int nsplit_max,
-                                                           int clusters, int* plan, int* list) {
-  extern __shared__ uint32_t bitmap[];
-  const int words = (T + 31) / 32;
-  int nact = 0;
-  if (words <= bitmap_words) {
-    for (int w = threadIdx.x; w < words; w += blockDim.x) {
-      uint32_t bits = 0;
-      const int t0 = w * 32, t1 = min(T, t0 + 32);
-      if (mask == nullptr) {
-        bits = (t1 - t0 == 32) ? 0xffffffffu : ((1u << (t1 - t0)) - 1u);
-      } else {
-        for (int t = t0; t < t1; ++t) bits |= (mask[t] != 0 ? 1u : 0u) << (t - t0);
-      }
-      bitmap[w] = bits;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      int t = 0;
-      while (t < T) {
-        // first loss token at or after t
-        int w = t >> 5;
-        uint32_t bits = bitmap[w] & (0xffffffffu << (t & 31));
-        while (bits == 0 && ++w < words) bits = bitmap[w];
-        if (bits == 0) break;
-        const int start = w * 32 + __ffs(bits) - 1;
-        list[nact++] = start;
-        t = start + 128;
-      }
-    }
-  } else if (threadIdx.x == 0) {
-    for (int b = 0; b * 128 < T; ++b) {
-      bool act = mask == nullptr;
-      for (int t = b * 128; t < min(T, b * 128 + 128) && !act; ++t) act = mask[t] != 0;
-      if (act) list[nact++] = b * 128;
-    }
+// One CTA.  Numbers the tokens that carry loss (m_t = 1) in packed order: compact row c of
+// token t = the count of loss tokens before t.  Tokens without loss have zero loss and zero
+// gradient, and no tile of any later kernel is spent on them: the tile kernels and the
+// contractions run over the compact rows 0..Tc-1, cut into blocks of 128.
+//   rows[c] = token of compact row c (0 for the padding rows Tc .. blocks*128-1)
+//   cidx[t] = compact row of token t, or -1
+//   plan    = {blocks, pairs of blocks, forward runs, Tc}
+__global__ void __launch_bounds__(1024) plan_rows_kernel(int T, const uint8_t* __restrict__ mask,
+                                                         int vtiles, int nsplit_max, int clusters,
+                                                         int* plan, int* rows, int* cidx) {
+  __shared__ int warp_tot[32];
+  __shared__ int total;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int per = (T + 1023) / 1024;                 // consecutive tokens per thread
+  const int t0 = min(T, static_cast<int>(threadIdx.x) * per), t1 = min(T, t0 + per);
+  int cnt = 0;
+  for (int t = t0; t < t1; ++t) cnt += (mask == nullptr || mask[t] != 0) ? 1 : 0;
+  // exclusive scan of cnt over the CTA
+  int incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
   }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_tot[lane], wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += v;
+    }
+    warp_tot[lane] = wi - w;                          // exclusive offsets of the warps
+    if (lane == 31) total = wi;
+  }
+  __syncthreads();
+  int c = warp_tot[warp] + incl - cnt;
+  for (int t = t0; t < t1; ++t) {
+    const bool on = mask == nullptr || mask[t] != 0;
+    cidx[t] = on ? c : -1;
+    if (on) rows[c++] = t;
+  }
+  const int tc = total, nact = (tc + 127) / 128, pairs = (nact + 1) / 2;
+  for (int i = tc + threadIdx.x; i < nact * 128; i += blockDim.x) rows[i] = 0;
   if (threadIdx.x == 0) {
-    const int pairs = (nact + 1) / 2;
     plan[0] = nact;
     plan[1] = pairs;
     plan[2] = choose_nsplit(pairs > 0 ? pairs : 1, vtiles, clusters, nsplit_max);
-    plan[3] = 0;
+    plan[3] = tc;
+  }
+}
+
+// Copies the hidden states of the compact rows next to each other (the padding rows of the last
+// block become zeros), so that the tile kernels and the dW contraction read them with plain
+// tiled TMA loads.  8 elements per thread.
+__global__ void __launch_bounds__(256) gather_hidden_rows_kernel(const __nv_bfloat16* __restrict__ H,
+                                                                 long long ldh, int d,
+                                                                 const int* __restrict__ plan,
+                                                                 const int* __restrict__ rows,
+                                                                 __nv_bfloat16* Hc) {
+  const int per_row = d / 8;
+  const long long n = static_cast<long long>(plan[0]) * 128 * per_row;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const int c = static_cast<int>(i / per_row), k = static_cast<int>(i % per_row) * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (c < plan[3]) v = *reinterpret_cast<const uint4*>(H + static_cast<size_t>(rows[c]) * ldh + k);
+    *reinterpret_cast<uint4*>(Hc + static_cast<size_t>(c) * d + k) = v;
   }
 }
 
 struct CombineParams {
   int T, d, V;
   const int* plan;        // plan[2] = forward runs; the partials hold 2 slots per run
+  const int* cidx;        // [T] compact row of a token (partials, lse2_*, coef* are indexed by it)
   const float* partials;  // [nslots][kPFields][T]
   const __nv_bfloat16* hidden;
   const __nv_bfloat16* weight;
@@ -136,25 +154,18 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
   const int nslots = 2 * p.plan[2];
   const bool on = p.loss_mask == nullptr || p.loss_mask[t] != 0;
   if (!on) {
-    // no loss and no gradient here; the token's block may not even have been visited
+    // no loss and no gradient here, and no compact row: nothing was computed for this token
     if (lane == 0) {
       p.kl[t] = 0.f;
       if (p.nll_s != nullptr) p.nll_s[t] = 0.f;
       if (p.nll_t != nullptr) p.nll_t[t] = 0.f;
-      // a huge log-sum-exp turns both probabilities of the gradient tile into exact zeros
-      p.lse2_a[t] = 1e30f;
-      p.lse2_b[t] = 1e30f;
-      p.coef[t] = 0.f;
-      if (p.coef_ce != nullptr) {
-        p.coef_ce[t] = 0.f;
-        p.lse2_b1[t] = 1e30f;
-      }
     }
     return;
   }
+  const int c = p.cidx[t];  // the token's compact row
   float ma = -INFINITY, mb = -INFINITY;
   for (int s = lane; s < nslots; s += 32) {
-    const float* q = p.partials + s * ss + t;
+    const float* q = p.partials + s * ss + c;
     ma = fmaxf(ma, q[kPMaxA * fs]);
     mb = fmaxf(mb, q[kPMaxB * fs]);
   }
@@ -162,7 +173,7 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
   mb = warp_max(mb);
   float sa = 0.f, cr = 0.f, sb = 0.f, sa1 = 0.f, sb1 = 0.f;
   for (int s = lane; s < nslots; s += 32) {
-    const float* q = p.partials + s * ss + t;
+    const float* q = p.partials + s * ss + c;
     const float da = q[kPMaxA * fs] - ma, db = q[kPMaxB * fs] - mb;
     const float fa = exp2f(da), fb = exp2f(db);
     sa = fmaf(q[kPSumA * fs], fa, sa);
@@ -219,12 +230,12 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
     p.kl[t] = on ? (kl < 0.f ? 0.f : kl) : 0.f;  // rounding may dip below 0; NaN stays NaN
     if (p.nll_s != nullptr) p.nll_s[t] = nll_s;
     if (p.nll_t != nullptr) p.nll_t[t] = nll_t;
-    p.lse2_a[t] = lse_a;
-    p.lse2_b[t] = lse_b;
-    p.coef[t] = on ? p.grad_scale * p.lambda / p.tau : 0.f;
+    p.lse2_a[c] = lse_a;
+    p.lse2_b[c] = lse_b;
+    p.coef[c] = p.grad_scale * p.lambda / p.tau;
     if (p.coef_ce != nullptr) {
-      p.coef_ce[t] = has_label ? p.grad_scale * (1.f - p.lambda) : 0.f;
-      p.lse2_b1[t] = kTauIsOne ? lse_b : mb * p.tau + log2f(sb1);
+      p.coef_ce[c] = has_label ? p.grad_scale * (1.f - p.lambda) : 0.f;
+      p.lse2_b1[c] = kTauIsOne ? lse_b : mb * p.tau + log2f(sb1);
     }
   }
 }
@@ -232,6 +243,7 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
 struct CombineTopkParams {
   int T, d, V, topk;
   const int* plan;        // plan[2] = forward runs; the partials hold 2 slots per run
+  const int* cidx;        // [T] compact row of a token (partials, lse2_b, coef*, tk_cp are indexed by it)
   const float* partials;  // [2*runs][kPFields][T]; only the student's fields are filled
   const __nv_bfloat16* hidden;
   const __nv_bfloat16* weight;
@@ -279,29 +291,23 @@ __global__ void __launch_bounds__(256) kd_combine_topk_kernel(const CombineTopkP
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (t >= p.T) return;
   const bool on = p.loss_mask == nullptr || p.loss_mask[t] != 0;
-  float* cp = p.tk_cp + static_cast<size_t>(t) * p.topk;
   if (!on) {
     if (lane == 0) {
       p.kl[t] = 0.f;
       if (p.nll_s != nullptr) p.nll_s[t] = 0.f;
-      p.lse2_b[t] = 1e30f;
-      p.coef[t] = 0.f;
-      if (p.coef_ce != nullptr) {
-        p.coef_ce[t] = 0.f;
-        p.lse2_b1[t] = 1e30f;
-      }
     }
-    for (int j = lane; j < p.topk; j += 32) cp[j] = 0.f;
     return;
   }
+  const int c = p.cidx[t];  // the token's compact row
+  float* cp = p.tk_cp + static_cast<size_t>(c) * p.topk;
   const int nslots = 2 * p.plan[2];
   const size_t fs = static_cast<size_t>(p.T), ss = static_cast<size_t>(kPFields) * fs;
   float mb = -INFINITY;
-  for (int s = lane; s < nslots; s += 32) mb = fmaxf(mb, p.partials[s * ss + kPMaxB * fs + t]);
+  for (int s = lane; s < nslots; s += 32) mb = fmaxf(mb, p.partials[s * ss + kPMaxB * fs + c]);
   mb = warp_max(mb);
   float sb = 0.f, sb1 = 0.f;
   for (int s = lane; s < nslots; s += 32) {
-    const float* q = p.partials + s * ss + t;
+    const float* q = p.partials + s * ss + c;
     const float db = q[kPMaxB * fs] - mb;
     sb = fmaf(q[kPSumB * fs], exp2f(db), sb);
     if (!kTauIsOne) sb1 = fmaf(q[kPSumB1 * fs], exp2f(db * p.tau), sb1);
@@ -345,11 +351,11 @@ __global__ void __launch_bounds__(256) kd_combine_topk_kernel(const CombineTopkP
     kl *= kLn2;
     p.kl[t] = kl < 0.f ? 0.f : kl;
     if (p.nll_s != nullptr) p.nll_s[t] = nll_s;
-    p.lse2_b[t] = lse_b;
-    p.coef[t] = coef;
+    p.lse2_b[c] = lse_b;
+    p.coef[c] = coef;
     if (p.coef_ce != nullptr) {
-      p.coef_ce[t] = has_label ? p.grad_scale * (1.f - p.lambda) : 0.f;
-      p.lse2_b1[t] = lse_b1;
+      p.coef_ce[c] = has_label ? p.grad_scale * (1.f - p.lambda) : 0.f;
+      p.lse2_b1[c] = lse_b1;
     }
   }
 }
@@ -440,22 +446,26 @@ __global__ void __launch_bounds__(256) select_kernel(
   if ((threadIdx.x & 31) == 0 && kept != 0) atomicAdd(n_keep, kept);
 }
 
-// fp32 [T, d] accumulator -> bf16 [T, ld] output, 8 elements per thread.
-__global__ void __launch_bounds__(256) f32_to_bf16_rows_kernel(const float* __restrict__ src, int T,
-                                                              int d, __nv_bfloat16* dst,
-                                                              long long ld) {
+// fp32 dH accumulator over the compact rows -> bf16 [T, ld] output by token; tokens without a
+// compact row (no loss) get zeros.  8 elements per thread.
+__global__ void __launch_bounds__(256) scatter_dhidden_kernel(const float* __restrict__ src,
+                                                             const int* __restrict__ cidx, int T, int d,
+                                                             __nv_bfloat16* dst, long long ld) {
   const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int per_row = d / 8;
   if (i >= static_cast<long long>(T) * per_row) return;
-  const int t = static_cast<int>(i / per_row), c = static_cast<int>(i % per_row) * 8;
-  const float4 a = *reinterpret_cast<const float4*>(src + static_cast<size_t>(t) * d + c);
-  const float4 b = *reinterpret_cast<const float4*>(src + static_cast<size_t>(t) * d + c + 4);
-  uint4 o;
-  o.x = pack_bf16x2(a.x, a.y);
-  o.y = pack_bf16x2(a.z, a.w);
-  o.z = pack_bf16x2(b.x, b.y);
-  o.w = pack_bf16x2(b.z, b.w);
-  *reinterpret_cast<uint4*>(dst + static_cast<size_t>(t) * ld + c) = o;
+  const int t = static_cast<int>(i / per_row), k = static_cast<int>(i % per_row) * 8;
+  const int c = cidx[t];
+  uint4 o = make_uint4(0u, 0u, 0u, 0u);
+  if (c >= 0) {
+    const float4 a = *reinterpret_cast<const float4*>(src + static_cast<size_t>(c) * d + k);
+    const float4 b = *reinterpret_cast<const float4*>(src + static_cast<size_t>(c) * d + k + 4);
+    o.x = pack_bf16x2(a.x, a.y);
+    o.y = pack_bf16x2(a.z, a.w);
+    o.z = pack_bf16x2(b.x, b.y);
+    o.w = pack_bf16x2(b.z, b.w);
+  }
+  *reinterpret_cast<uint4*>(dst + static_cast<size_t>(t) * ld + k) = o;
 }
 
 }  // namespace npd
