@@ -9,9 +9,11 @@
 // and the hidden states be read as they lie in memory, with no transposes.
 //
 // One launch runs one or two such problems.  With two, the CTA pairs first take the
-// (long) units of problem 0 and then the (short, split-K) units of problem 1, dealt
-// so that every pair ends at about the same time; this is how the dW and dH products
-// of one vocabulary chunk share a launch without a tail in between.
+// units (whole tiles) of problem 0 round robin; problem 1 is then laid out as one long line
+// of (tile, k-step) positions and every pair gets the stretch of that line that brings it to
+// the same total number of k-steps as all the others (a stretch may start and end in the
+// middle of a tile: the pieces are added with fp32 atomics).  This is how the dW and dH
+// products of one vocabulary chunk share a launch and end together.
 //
 // Two CTAs on neighbouring SMs (a cluster of 2) work as a pair on a 256 x 512 output tile
 // with tcgen05 .cta_group::2 (two M=256, N=256 accumulators that share the A operand): per
@@ -43,6 +45,8 @@ struct GemmProblem {
   // batch, nblocks[0] blocks of 128):
   int dyn_m;       // M = 128 * nblocks[0]
   int dyn_k;       // K = 128 * nblocks[0]
+  int stream_k;    // problem 1 only: cut along the (tile, k-step) line as described above
+                   // (needs out_reduce and k_splits = 1)
 };
 
 struct GemmParams {
@@ -50,13 +54,6 @@ struct GemmParams {
   int nprob;           // 1 or 2
   const int* nblocks;  // device; read only when a problem has dyn_m / dyn_k
   int* status;         // device status word
-};
-
-// How the units of the one or two problems are dealt to the CTA pairs.
-struct GemmSched {
-  int units[2];    // work units of each problem (tiles x k_splits); units[1] = 0 for a single problem
-  int q0, rem0;    // units[0] = q0 * pairs + rem0
-  int extra1;      // units of problem 1 that each pair WITHOUT a remainder unit of problem 0 takes first
 };
 
 namespace gemm_cfg {
@@ -79,76 +76,93 @@ constexpr int OFF_BAR = OFF_OUT + 2 * OUT_BYTES;
 constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;  // + barriers + alignment
 }  // namespace gemm_cfg
 
-// The i-th unit of CTA pair c out of C.  Problem-0 units go round robin.  The pairs that got
-// one unit fewer of problem 0 (c >= rem0) make up for it with `extra1` units of problem 1;
-// the rest of problem 1 goes round robin over all pairs.
-__host__ __device__ inline bool gemm_unit_at(const GemmSched& p, int c, int C, int i, int& prob, int& v) {
-  const int n0 = p.q0 + (c < p.rem0 ? 1 : 0);
-  if (i < n0) {
-    prob = 0;
-    v = c + i * C;
-    return true;
-  }
-  prob = 1;
-  int j = i - n0;
-  int base = 0;
-  if (p.rem0 > 0) {
-    const int nb = C - p.rem0;
-    base = p.extra1 * nb;
-    if (c >= p.rem0) {
-      if (j < p.extra1) {
-        v = j * nb + (c - p.rem0);
-        return v < p.units[1];
-      }
-      j -= p.extra1;
-    }
-  }
-  v = base + j * C + c;
-  return v < p.units[1];
-}
-
-__host__ __device__ inline int gemm_unit_ksteps(const GemmProblem& g) {
-  const int kt = (g.K + 63) / 64;
-  const int per = (kt + g.k_splits - 1) / g.k_splits;
-  return per > 0 ? per : 1;
-}
-// Resolves the device-side dimensions and deals the units to C pairs.
-__device__ __forceinline__ void gemm_setup(const GemmParams& p, int C, GemmProblem (&pr)[2], GemmSched& sc) {
-  pr[0] = p.pr[0];
-  pr[1] = p.pr[1];
-#pragma unroll
-  for (int i = 0; i < 2; ++i) {
-    if (pr[i].dyn_m) pr[i].M = 128 * __ldg(p.nblocks);
-    if (pr[i].dyn_k) pr[i].K = 128 * __ldg(p.nblocks);
-    const int tiles = ((pr[i].M + 255) / 256) * ((pr[i].N + 511) / 512);
-    sc.units[i] = i < p.nprob ? tiles * pr[i].k_splits : 0;
-  }
-  sc.q0 = sc.units[0] / C;
-  sc.rem0 = sc.units[0] % C;
-  sc.extra1 = 0;
-  if (sc.units[1] > 0 && sc.rem0 > 0) {
-    const int c0 = gemm_unit_ksteps(pr[0]), c1 = gemm_unit_ksteps(pr[1]);
-    const int want = (c0 + c1 / 2) / c1, can = sc.units[1] / (C - sc.rem0);
-    sc.extra1 = want < can ? want : can;
-  }
-}
-
 struct GemmUnit {
   int m0, n0, kt0, kt1;  // pair-tile origin and k-tile range
   int ns;                // accumulators in use: 2, or 1 when the tile's second 256 columns lie beyond N
 };
-__device__ __forceinline__ GemmUnit gemm_decode(const GemmProblem& g, int v) {
+// Tile `tile` (n fastest) of a problem, k-tiles [kt0, kt1).
+__device__ __forceinline__ GemmUnit gemm_tile_unit(const GemmProblem& g, int tile, int kt0, int kt1) {
   using namespace gemm_cfg;
-  const int tiles_m = (g.M + PM - 1) / PM, tiles_n = (g.N + BN - 1) / BN, ktiles = (g.K + BK - 1) / BK;
-  const int ks = v / (tiles_n * tiles_m);
+  const int tiles_n = (g.N + BN - 1) / BN;
   GemmUnit u;
-  u.n0 = (v % tiles_n) * BN;
-  u.m0 = ((v / tiles_n) % tiles_m) * PM;
-  u.kt0 = static_cast<int>(static_cast<long long>(ktiles) * ks / g.k_splits);
-  u.kt1 = static_cast<int>(static_cast<long long>(ktiles) * (ks + 1) / g.k_splits);
+  u.n0 = (tile % tiles_n) * BN;
+  u.m0 = (tile / tiles_n) * PM;
+  u.kt0 = kt0;
+  u.kt1 = kt1;
   u.ns = (g.N - u.n0 > BNS) ? 2 : 1;
   return u;
 }
+
+// The sequence of units of one CTA pair.  Every role of both CTAs walks the same sequence.
+struct GemmWalk {
+  GemmProblem pr[2];
+  int c, C;            // this pair and the number of pairs
+  int tiles[2], ksteps[2];
+  int i;               // units taken so far in the round-robin phases
+  long long pos, end;  // problem 1 with stream_k: this pair's stretch of the (tile, k-step) line
+
+  __device__ __forceinline__ void init(const GemmParams& p, int c_, int C_) {
+    using namespace gemm_cfg;
+    c = c_;
+    C = C_;
+    i = 0;
+    pos = end = 0;
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      pr[q] = p.pr[q];
+      if (pr[q].dyn_m) pr[q].M = 128 * __ldg(p.nblocks);
+      if (pr[q].dyn_k) pr[q].K = 128 * __ldg(p.nblocks);
+      tiles[q] = q < p.nprob ? ((pr[q].M + PM - 1) / PM) * ((pr[q].N + BN - 1) / BN) : 0;
+      ksteps[q] = (pr[q].K + BK - 1) / BK;
+    }
+    if (tiles[1] > 0 && pr[1].stream_k && ksteps[1] > 0) {
+      // k-steps of problem 0 this pair and its neighbours carry (units go round robin)
+      const int units0 = tiles[0] * pr[0].k_splits, q0 = units0 / C, rem0 = units0 % C;
+      const double c0 = static_cast<double>((ksteps[0] + pr[0].k_splits - 1) / pr[0].k_splits);
+      const double line = static_cast<double>(tiles[1]) * ksteps[1];
+      const double target = (units0 * c0 + line) / C;
+      // pairs 0..rem0-1 hold one more unit of problem 0 and get the shorter stretch sa
+      double sa = target - (q0 + 1) * c0;
+      sa = sa > 0.0 ? sa : 0.0;
+      const double sb = rem0 < C ? (line - rem0 * sa) / (C - rem0) : 0.0;
+      auto prefix = [&](int k) { return k <= rem0 ? k * sa : rem0 * sa + (k - rem0) * sb; };
+      pos = static_cast<long long>(prefix(c) + 0.5);
+      end = c + 1 == C ? static_cast<long long>(tiles[1]) * ksteps[1] : static_cast<long long>(prefix(c + 1) + 0.5);
+    }
+  }
+
+  __device__ __forceinline__ bool next(int& prob, GemmUnit& u) {
+    const int units0 = tiles[0] * pr[0].k_splits;
+    const int mine0 = units0 / C + (c < units0 % C ? 1 : 0);
+    if (i < mine0) {
+      const int v = c + i * C, ks = v / tiles[0];
+      prob = 0;
+      u = gemm_tile_unit(pr[0], v % tiles[0],
+                         static_cast<int>(static_cast<long long>(ksteps[0]) * ks / pr[0].k_splits),
+                         static_cast<int>(static_cast<long long>(ksteps[0]) * (ks + 1) / pr[0].k_splits));
+      ++i;
+      return true;
+    }
+    prob = 1;
+    if (pr[1].stream_k) {
+      if (pos >= end) return false;
+      const int tile = static_cast<int>(pos / ksteps[1]), k0 = static_cast<int>(pos % ksteps[1]);
+      const long long left = end - pos;
+      const int len = left < ksteps[1] - k0 ? static_cast<int>(left) : ksteps[1] - k0;
+      u = gemm_tile_unit(pr[1], tile, k0, k0 + len);
+      pos += len;
+      return true;
+    }
+    const int v = c + (i - mine0) * C;
+    if (v >= tiles[1] * pr[1].k_splits) return false;
+    const int ks = v / tiles[1];
+    u = gemm_tile_unit(pr[1], v % tiles[1],
+                       static_cast<int>(static_cast<long long>(ksteps[1]) * ks / pr[1].k_splits),
+                       static_cast<int>(static_cast<long long>(ksteps[1]) * (ks + 1) / pr[1].k_splits));
+    ++i;
+    return true;
+  }
+};
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(gemm_cfg::THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_constant__ CUtensorMap tmap_b0,
@@ -201,20 +215,19 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
   const uint32_t full_leader = mapa_shared(full0, 0);
   const uint32_t tempty_leader = mapa_shared(tempty, 0);
 
-  // every role resolves the same problems and the same deal of units
-  GemmProblem pr[2];
-  GemmSched sc;
-  gemm_setup(p, num_clusters, pr, sc);
+  // every role resolves the same problems and walks the same sequence of units
+  GemmWalk walk;
+  walk.init(p, cluster_id, num_clusters);
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      int prob, v;
-      for (int i = 0; ok && gemm_unit_at(sc, cluster_id, num_clusters, i, prob, v); ++i) {
-        const GemmProblem& g = prob ? pr[1] : pr[0];
-        const GemmUnit u = gemm_decode(g, v);
+      int prob;
+      GemmUnit u;
+      while (ok && walk.next(prob, u)) {
+        const GemmProblem& g = prob ? walk.pr[1] : walk.pr[0];
         const CUtensorMap* ta = prob ? &tmap_a1 : &tmap_a0;
         const CUtensorMap* tb = prob ? &tmap_b1 : &tmap_b0;
         const int m0 = u.m0 + static_cast<int>(rank) * BM;          // this CTA's A rows
@@ -260,10 +273,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
     if (rank == 0 && lane == 0) {
       uint32_t it = 0, tile = 0;
       bool ok = true;
-      int prob, v;
-      for (int i = 0; ok && gemm_unit_at(sc, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
-        const GemmProblem& g = prob ? pr[1] : pr[0];
-        const GemmUnit u = gemm_decode(g, v);
+      int prob;
+      GemmUnit u;
+      for (; ok && walk.next(prob, u); ++tile) {
+        const GemmProblem& g = prob ? walk.pr[1] : walk.pr[0];
         const uint32_t idesc = umma_idesc_bf16(PM, BNS, g.a_mn != 0, g.b_mn != 0);
         // the accumulators are free once every epilogue warp of the pair has read the last tile
         if (!(ok = mbar_wait(tempty, (tile & 1) ^ 1, abort_flag))) break;
@@ -303,10 +316,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
     const int bar_id = 1 + grp;
     uint32_t tile = 0;
     bool ok = true;
-    int prob, v;
-    for (int i = 0; ok && gemm_unit_at(sc, cluster_id, num_clusters, i, prob, v); ++i, ++tile) {
-      const GemmProblem& g = prob ? pr[1] : pr[0];
-      const GemmUnit u = gemm_decode(g, v);
+    int prob;
+    GemmUnit u;
+    for (; ok && walk.next(prob, u); ++tile) {
+      const GemmProblem& g = prob ? walk.pr[1] : walk.pr[0];
       const CUtensorMap* to = prob ? &tmap_o1 : &tmap_o0;
       const int m0 = u.m0 + static_cast<int>(rank) * BM;
       const bool rows_inside = m0 < g.M;          // else this CTA's 128 rows lie beyond M: nothing to store

@@ -73,7 +73,6 @@ struct Plan {
   int nsplit_max;     // upper bound of the forward's vocabulary runs (the device picks the number)
   int chunk_cols;     // vocabulary columns per gradient chunk (multiple of 256)
   int nchunks;
-  int dh_ksplits;     // split-K of the dH product of a full chunk
   bool grads;
   size_t off_status, off_plan, off_rows, off_cidx, off_hc, off_partials, off_lse_a, off_lse_b, off_coef, off_coef_ce,
       off_lse_b1, off_tkcp, off_g, off_dh, total;
@@ -102,13 +101,6 @@ int make_plan(const npd_kd_args* a, int sms, Plan* pl) {
   pl->chunk_cols = chunk_tiles * 256;
   pl->nchunks = (pl->vtiles + chunk_tiles - 1) / chunk_tiles;
   const int cc = pl->chunk_cols;
-  // dH = G W is cut along the chunk's columns (split-K, partial products added with fp32
-  // atomics) only as far as it takes to give every CTA pair about 8 units, and never into
-  // units shorter than 48 k-steps: short units pay the accumulator drain too often.
-  const int ksteps_h = cc / 64;
-  const long long tiles_h = static_cast<long long>((pl->row_blocks + 1) / 2) * ((a->d + 511) / 512);
-  const int want = static_cast<int>((8ll * pl->clusters + tiles_h - 1) / tiles_h);
-  pl->dh_ksplits = std::max(1, std::min(want, ksteps_h / 48));
   size_t off = 0;
   pl->off_status = off;
   off += 1024;
@@ -513,7 +505,8 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     pr[1].K = cols;
     pr[1].a_mn = 0;
     pr[1].b_mn = 1;
-    pr[1].k_splits = std::max(1, std::min(pl.dh_ksplits, (cols + 63) / 64));
+    pr[1].k_splits = 1;
+    pr[1].stream_k = 1;
     pr[1].out_f32 = 1;
     pr[1].out_reduce = 1;
     const __nv_bfloat16* w_rows = static_cast<const __nv_bfloat16*>(a->weight) + static_cast<size_t>(col0) * a->ldw;
