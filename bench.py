@@ -237,7 +237,7 @@ def run_ours(args):
     from paper_2605_05940_b200 import binding as B, build as npd_build, synth_inputs as syn
     npd_build.build()
 
-    wl = dict(WORKLOAD, T=args.T)
+    wl = dict(WORKLOAD, T=args.T, d=args.d)
     # every rank draws its own batch (independent replicas)
     b = syn.config2_1b(device=dev, T=wl["T"], d=wl["d"], V=wl["V"], seed_base=2000 + 100 * rank)
     topk = {}
@@ -367,6 +367,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--T", type=int, default=WORKLOAD["T"],
                     help="packed tokens; anything but the default is a profiling case, not a bench value")
+    ap.add_argument("--d", type=int, default=WORKLOAD["d"], help="hidden size; as for --T")
     ap.add_argument("--grad-chunk-cols", type=int, default=0, help="0 = library default")
     ap.add_argument("--teacher", default="dense", choices=["dense", "topk"],
                     help="dense = the benchmark's workload; topk = k=10 stored logits (implies --no-e2e)")
