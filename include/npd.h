@@ -155,14 +155,13 @@ int npd_phase_count(const npd_kd_args* args, int32_t* out_groups, int32_t* out_c
  * is a HOST struct holding device pointers.  Enqueues on `cuda_stream`.
  *
  * Tokens with loss_mask 0 have kl = nll = 0 and no gradient by definition; the kernels
- * cover the tokens that carry loss with 128-row blocks (found on the device from
- * loss_mask) and spend no work on the rest, so a batch with long masked prompts costs
- * proportionally less.  Every output element is written all the same (zeros where
- * nothing is computed).
+ * compact the tokens that carry loss (on the device, from loss_mask) and spend no work
+ * on the rest, so a batch with 30 % masked prompt tokens costs 30 % less.  Every output
+ * element is written all the same (zeros where nothing is computed).
  *
  * kl, nll_*, and d_weight are bitwise reproducible from run to run.  d_hidden is summed
- * over vocabulary chunks with fp32 atomic adds whose order is not fixed: its last bits
- * may differ between runs. */
+ * over vocabulary chunks with fp32 atomic adds whose order is not fixed: a few of its
+ * bf16 elements may round differently between runs. */
 int npd_kd_fwd_bwd(const npd_kd_args* args, void* cuda_stream);
 
 /*
@@ -271,7 +270,7 @@ int npd_last_launch_count(void);
  * passes all inputs and the kl / nll_* outputs.  A problem whose scratch
  * (npd_workspace_bytes of the same forward-only arguments) exceeds
  * NPD_STATIC_SCRATCH_BYTES is refused with NPD_EWORKSPACE before anything is launched;
- * c2's forward (T=8192, V=151,936) needs about 17 MB.  The call makes no cudaMalloc,
+ * c2's forward (T=8192, d=1536, V=151,936) needs about 40 MB.  The call makes no cudaMalloc,
  * cudaFree or other allocating call.
  *
  * The first call on each device looks up the array's device address (with that device
