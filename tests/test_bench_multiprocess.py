@@ -25,12 +25,18 @@ def _torchrun(script_and_args, timeout):
 
 
 def _json_lines(text):
-    out = []
-    for ln in text.splitlines():
-        ln = ln.strip()
-        if ln.startswith("{") and ln.endswith("}"):
-            out.append(json.loads(ln))
-    return out
+    """Every JSON object in the output (two ranks may write to the same line)."""
+    dec, out, i = json.JSONDecoder(), [], 0
+    while True:
+        i = text.find("{", i)
+        if i < 0:
+            return out
+        try:
+            obj, end = dec.raw_decode(text, i)
+            out.append(obj)
+            i = end
+        except json.JSONDecodeError:
+            i += 1
 
 
 def test_rank_plumbing_world_size_2():
