@@ -173,7 +173,10 @@ int npd_kd_fwd_bwd(const npd_kd_args* args, void* cuda_stream);
  * nll_student, nll_teacher).  The weight is a resident parameter and the two
  * gradients stay on the device: host->weight, d_hidden, d_weight are ignored.
  * The call copies the inputs in, runs npd_kd_fwd_bwd(dev) and copies the
- * per-token outputs back, all asynchronously on `cuda_stream`.
+ * per-token outputs back, all asynchronously on `cuda_stream`.  Of hidden and teacher
+ * (or the top-k arrays) only the rows of tokens with loss_mask != 0 are copied (the host
+ * mask is read during the call): the kernels never read the other rows, and the staging
+ * buffers keep whatever they held there.
  */
 int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* cuda_stream);
 
@@ -252,6 +255,10 @@ const char* npd_strerror(int status);
 /* HOST.  Number of kernel launches the last npd_kd_fwd_bwd call on this thread
  * enqueued (for launch accounting in benchmarks). */
 int npd_last_launch_count(void);
+
+/* HOST.  Bytes the last npd_kd_fwd_bwd_host call on this thread copied host-to-device and
+ * device-to-host. */
+int npd_last_copy_bytes(int64_t* h2d_bytes, int64_t* d2h_bytes);
 
 /*
  * Forward pass without any workspace from the caller.  (The paper has no counterpart

@@ -30,7 +30,7 @@ NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32 =
 
 EXPORTS = ("npd_workspace_bytes", "npd_phase_count", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
            "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16",
-           "npd_kd_forward_noalloc", "npd_pack_sequences")
+           "npd_kd_forward_noalloc", "npd_pack_sequences", "npd_last_copy_bytes")
 NPD_STATIC_SCRATCH_BYTES = 48 * 1024 * 1024
 
 
@@ -82,6 +82,7 @@ def lib() -> C.CDLL:
                                  + [C.c_void_p] * 6)
         l.npd_last_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
         l.npd_last_launch_count.argtypes = []
+        l.npd_last_copy_bytes.argtypes = [C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         l.npd_kd_forward_noalloc.argtypes = [C.POINTER(npd_kd_args), C.c_void_p, C.POINTER(C.c_int32)]
         l.npd_pack_sequences.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_int32] + [C.c_void_p] * 6
         l.npd_gemm_bf16.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int32,
@@ -185,6 +186,13 @@ def npd_last_status(workspace: torch.Tensor, stream=None) -> int:
 
 def npd_last_launch_count() -> int:
     return lib().npd_last_launch_count()
+
+
+def npd_last_copy_bytes():
+    """(host-to-device, device-to-host) bytes of the last npd_kd_fwd_bwd_host call on this thread."""
+    a, b = C.c_int64(0), C.c_int64(0)
+    _check(lib().npd_last_copy_bytes(C.byref(a), C.byref(b)), "npd_last_copy_bytes")
+    return a.value, b.value
 
 
 def npd_segment_stats(cu_seqlens, loss_mask, labels, kl, nll_student, nll_teacher, *,

@@ -23,6 +23,7 @@ namespace {
 using namespace npd;
 
 thread_local int g_launches = 0;
+thread_local long long g_h2d_bytes = 0, g_d2h_bytes = 0;  // of the last npd_kd_fwd_bwd_host call
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -280,6 +281,13 @@ const char* npd_strerror(int status) {
 }
 
 int npd_last_launch_count(void) { return g_launches; }
+
+int npd_last_copy_bytes(int64_t* h2d_bytes, int64_t* d2h_bytes) {
+  if (h2d_bytes == nullptr || d2h_bytes == nullptr) return NPD_EINVAL;
+  *h2d_bytes = g_h2d_bytes;
+  *d2h_bytes = g_d2h_bytes;
+  return NPD_OK;
+}
 
 int npd_workspace_bytes(const npd_kd_args* args, size_t* out_bytes) {
   if (out_bytes == nullptr) return NPD_EINVAL;
@@ -555,36 +563,69 @@ int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* c
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t T = dev->T;
   bool ok = true;
-  ok &= cudaMemcpy2DAsync(const_cast<void*>(dev->hidden), dev->ldh * 2, host->hidden, host->ldh * 2,
-                          static_cast<size_t>(dev->d) * 2, T, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (dev->topk > 0) {
-    const size_t n = T * static_cast<size_t>(dev->topk);
-    ok &= cudaMemcpyAsync(const_cast<float*>(dev->topk_values), host->topk_values, n * sizeof(float),
-                          cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->topk_indices), host->topk_indices, n * sizeof(int32_t),
-                          cudaMemcpyHostToDevice, st) == cudaSuccess;
-  } else {
-    ok &= cudaMemcpy2DAsync(const_cast<void*>(dev->teacher), dev->ldt * 2, host->teacher, host->ldt * 2,
-                            static_cast<size_t>(dev->V) * 2, T, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  g_h2d_bytes = g_d2h_bytes = 0;
+  // Rows of tokens without loss are never read by the kernels, so only the stretches of rows
+  // that carry loss are copied (a batch with masked prompts moves that much less over PCIe).
+  // With a mask that would take too many separate copies, everything is copied.
+  std::vector<std::pair<size_t, size_t>> runs;  // [first row, end row)
+  const bool have_mask = host->loss_mask != nullptr && dev->loss_mask != nullptr;
+  if (have_mask) {
+    size_t t = 0;
+    while (t < T && runs.size() <= 1024) {
+      while (t < T && host->loss_mask[t] == 0) ++t;
+      const size_t a = t;
+      while (t < T && host->loss_mask[t] != 0) ++t;
+      if (t > a) runs.emplace_back(a, t);
+    }
   }
-  if (dev->cu_seqlens != nullptr && host->cu_seqlens != nullptr)
+  if (!have_mask || runs.size() > 1024) runs.assign(1, std::make_pair(size_t{0}, T));
+  auto copy_rows = [&](const void* dst, long long ldd, const void* src, long long lds, size_t row_bytes,
+                       size_t esize) {
+    for (const auto& r : runs) {
+      const size_t n = r.second - r.first;
+      ok &= cudaMemcpy2DAsync(static_cast<char*>(const_cast<void*>(dst)) + r.first * ldd * esize, ldd * esize,
+                              static_cast<const char*>(src) + r.first * lds * esize, lds * esize, row_bytes,
+                              n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+      g_h2d_bytes += static_cast<long long>(row_bytes * n);
+    }
+  };
+  copy_rows(dev->hidden, dev->ldh, host->hidden, host->ldh, static_cast<size_t>(dev->d) * 2, 2);
+  if (dev->topk > 0) {
+    copy_rows(dev->topk_values, dev->topk, host->topk_values, dev->topk, sizeof(float) * dev->topk, sizeof(float));
+    copy_rows(dev->topk_indices, dev->topk, host->topk_indices, dev->topk, sizeof(int32_t) * dev->topk,
+              sizeof(int32_t));
+  } else {
+    copy_rows(dev->teacher, dev->ldt, host->teacher, host->ldt, static_cast<size_t>(dev->V) * 2, 2);
+  }
+  if (dev->cu_seqlens != nullptr && host->cu_seqlens != nullptr) {
     ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->cu_seqlens), host->cu_seqlens,
                           sizeof(int32_t) * (dev->S + 1), cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (dev->loss_mask != nullptr && host->loss_mask != nullptr)
+    g_h2d_bytes += static_cast<long long>(sizeof(int32_t)) * (dev->S + 1);
+  }
+  if (have_mask) {
     ok &= cudaMemcpyAsync(const_cast<uint8_t*>(dev->loss_mask), host->loss_mask, T,
                           cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (dev->labels != nullptr && host->labels != nullptr)
+    g_h2d_bytes += static_cast<long long>(T);
+  }
+  if (dev->labels != nullptr && host->labels != nullptr) {
     ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->labels), host->labels, sizeof(int32_t) * T,
                           cudaMemcpyHostToDevice, st) == cudaSuccess;
+    g_h2d_bytes += static_cast<long long>(sizeof(int32_t) * T);
+  }
   if (!ok) return NPD_ECUDA;
   if ((rc = npd_kd_fwd_bwd(dev, cuda_stream)) != NPD_OK) return rc;
   ok &= cudaMemcpyAsync(host->kl, dev->kl, sizeof(float) * T, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (host->nll_student != nullptr && dev->nll_student != nullptr)
+  g_d2h_bytes += static_cast<long long>(sizeof(float) * T);
+  if (host->nll_student != nullptr && dev->nll_student != nullptr) {
     ok &= cudaMemcpyAsync(host->nll_student, dev->nll_student, sizeof(float) * T,
                           cudaMemcpyDeviceToHost, st) == cudaSuccess;
-  if (host->nll_teacher != nullptr && dev->nll_teacher != nullptr)
+    g_d2h_bytes += static_cast<long long>(sizeof(float) * T);
+  }
+  if (host->nll_teacher != nullptr && dev->nll_teacher != nullptr) {
     ok &= cudaMemcpyAsync(host->nll_teacher, dev->nll_teacher, sizeof(float) * T,
                           cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    g_d2h_bytes += static_cast<long long>(sizeof(float) * T);
+  }
   return ok ? NPD_OK : NPD_ECUDA;
 }
 
