@@ -243,6 +243,19 @@ def test_loss_tokens_in_scattered_stretches(ranges):
     check_full_parity(b, step)
 
 
+def test_many_blocks_long_batch_small_vocabulary():
+    # 70,000 packed tokens: hundreds of row blocks (an odd number of them), several tokens per
+    # planning thread, one ragged vocabulary tile; small d and V keep the oracle quick
+    b = syn.scaled("c2", device=DEV, T=70000, d=64, V=520, seed_base=21, min_len=30, max_len=3000)
+    step = run_step(b, dw_dtype=torch.float32)
+    kl, ns, nt = check_full_parity(b, step)
+    check_stats_and_select(b, step, kl, ns, nt)
+    # and with every token carrying loss (no mask at all)
+    b.loss_mask[:] = 1
+    step = run_step(b, dw_dtype=torch.float32)
+    check_full_parity(b, step)
+
+
 def test_optional_inputs_may_be_null():
     b = _mini()
     H, W, Z, y, m = oracle_inputs(b)
