@@ -181,6 +181,17 @@ int npd_kd_fwd_bwd(const npd_kd_args* args, void* cuda_stream);
 int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* cuda_stream);
 
 /*
+ * The same with the copies in on a stream of their own.  The copies wait for everything
+ * queued so far on `cuda_stream` (the last user of the staging buffers in `dev`), the kernels
+ * wait for the copies; the copies back run on `cuda_stream`.  A caller that alternates between
+ * two sets of staging buffers, each with its own `cuda_stream`, and gives every call the same
+ * `copy_stream`, gets the copies of step i+1 under the kernels of step i, one transfer at a
+ * time on the link.  Creates and releases two CUDA events per call (no device memory).
+ */
+int npd_kd_fwd_bwd_host_streams(const npd_kd_args* host, const npd_kd_args* dev, void* copy_stream,
+                                void* cuda_stream);
+
+/*
  * Per-sample statistics for the Delta-IFD filter (the sums behind Eq. 3):
  *   kl_sum[s]    = sum_{t in s} m_t kl[t]
  *   nll_s_sum[s] = sum_{t in s} m_t [y_t>=0] nll_student[t]     (same for teacher)

@@ -30,7 +30,8 @@ NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32 =
 
 EXPORTS = ("npd_workspace_bytes", "npd_phase_count", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
            "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16",
-           "npd_kd_forward_noalloc", "npd_pack_sequences", "npd_last_copy_bytes")
+           "npd_kd_forward_noalloc", "npd_pack_sequences", "npd_last_copy_bytes",
+           "npd_kd_fwd_bwd_host_streams")
 NPD_STATIC_SCRATCH_BYTES = 48 * 1024 * 1024
 
 
@@ -77,6 +78,8 @@ def lib() -> C.CDLL:
         l.npd_kd_fwd_bwd.argtypes = [C.POINTER(npd_kd_args), C.c_void_p]
         l.npd_phase_count.argtypes = [C.POINTER(npd_kd_args), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         l.npd_kd_fwd_bwd_host.argtypes = [C.POINTER(npd_kd_args), C.POINTER(npd_kd_args), C.c_void_p]
+        l.npd_kd_fwd_bwd_host_streams.argtypes = [C.POINTER(npd_kd_args), C.POINTER(npd_kd_args), C.c_void_p,
+                                                  C.c_void_p]
         l.npd_segment_stats.argtypes = [C.c_int32, C.c_int32] + [C.c_void_p] * 13
         l.npd_select.argtypes = ([C.c_int32] + [C.c_void_p] * 5 + [C.c_int32, C.c_float, C.c_float, C.c_int32]
                                  + [C.c_void_p] * 6)
@@ -166,6 +169,11 @@ def npd_kd_fwd_bwd(args: npd_kd_args, stream=None) -> None:
 
 def npd_kd_fwd_bwd_host(host: npd_kd_args, dev: npd_kd_args, stream=None) -> None:
     _check(lib().npd_kd_fwd_bwd_host(C.byref(host), C.byref(dev), _stream(stream)), "npd_kd_fwd_bwd_host")
+
+
+def npd_kd_fwd_bwd_host_streams(host: npd_kd_args, dev: npd_kd_args, copy_stream, stream=None) -> None:
+    _check(lib().npd_kd_fwd_bwd_host_streams(C.byref(host), C.byref(dev), _stream(copy_stream), _stream(stream)),
+           "npd_kd_fwd_bwd_host_streams")
 
 
 def npd_kd_forward_noalloc(args: npd_kd_args, stream=None, want_status: bool = False):

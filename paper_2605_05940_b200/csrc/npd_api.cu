@@ -552,6 +552,11 @@ int npd_phase_count(const npd_kd_args* args, int32_t* out_groups, int32_t* out_c
 }
 
 int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* cuda_stream) {
+  return npd_kd_fwd_bwd_host_streams(host, dev, cuda_stream, cuda_stream);
+}
+
+int npd_kd_fwd_bwd_host_streams(const npd_kd_args* host, const npd_kd_args* dev, void* copy_stream,
+                                void* cuda_stream) {
   if (host == nullptr || dev == nullptr || host->size != sizeof(npd_kd_args)) return NPD_EINVAL;
   int rc = check_args(dev, true);
   if (rc != NPD_OK) return rc;
@@ -560,10 +565,22 @@ int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* c
   if (dev->topk > 0 ? (host->topk_values == nullptr || host->topk_indices == nullptr)
                     : (host->teacher == nullptr))
     return NPD_EINVAL;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);  // kernels and the copies back
+  cudaStream_t cs = static_cast<cudaStream_t>(copy_stream);  // the copies in
   const size_t T = dev->T;
   bool ok = true;
   g_h2d_bytes = g_d2h_bytes = 0;
+  // With a copy stream of its own: the copies in start once everything queued so far on the
+  // compute stream (the last user of these staging buffers) is done, and the kernels start once
+  // the copies are.  Copies of different calls queue up behind each other on the copy stream
+  // instead of sharing the link, so a call's kernels overlap the next call's copies.
+  const bool two_streams = cs != st;
+  cudaEvent_t ev = nullptr;
+  if (two_streams) {
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return NPD_ECUDA;
+    ok &= cudaEventRecord(ev, st) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(cs, ev, 0) == cudaSuccess;
+  }
   // Rows of tokens without loss are never read by the kernels, so only the stretches of rows
   // that carry loss are copied (a batch with masked prompts moves that much less over PCIe).
   // With a mask that would take too many separate copies, everything is copied.
@@ -585,7 +602,7 @@ int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* c
       const size_t n = r.second - r.first;
       ok &= cudaMemcpy2DAsync(static_cast<char*>(const_cast<void*>(dst)) + r.first * ldd * esize, ldd * esize,
                               static_cast<const char*>(src) + r.first * lds * esize, lds * esize, row_bytes,
-                              n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+                              n, cudaMemcpyHostToDevice, cs) == cudaSuccess;
       g_h2d_bytes += static_cast<long long>(row_bytes * n);
     }
   };
@@ -599,18 +616,23 @@ int npd_kd_fwd_bwd_host(const npd_kd_args* host, const npd_kd_args* dev, void* c
   }
   if (dev->cu_seqlens != nullptr && host->cu_seqlens != nullptr) {
     ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->cu_seqlens), host->cu_seqlens,
-                          sizeof(int32_t) * (dev->S + 1), cudaMemcpyHostToDevice, st) == cudaSuccess;
+                          sizeof(int32_t) * (dev->S + 1), cudaMemcpyHostToDevice, cs) == cudaSuccess;
     g_h2d_bytes += static_cast<long long>(sizeof(int32_t)) * (dev->S + 1);
   }
   if (have_mask) {
     ok &= cudaMemcpyAsync(const_cast<uint8_t*>(dev->loss_mask), host->loss_mask, T,
-                          cudaMemcpyHostToDevice, st) == cudaSuccess;
+                          cudaMemcpyHostToDevice, cs) == cudaSuccess;
     g_h2d_bytes += static_cast<long long>(T);
   }
   if (dev->labels != nullptr && host->labels != nullptr) {
     ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->labels), host->labels, sizeof(int32_t) * T,
-                          cudaMemcpyHostToDevice, st) == cudaSuccess;
+                          cudaMemcpyHostToDevice, cs) == cudaSuccess;
     g_h2d_bytes += static_cast<long long>(sizeof(int32_t) * T);
+  }
+  if (two_streams) {
+    ok &= cudaEventRecord(ev, cs) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(st, ev, 0) == cudaSuccess;
+    cudaEventDestroy(ev);  // released once the recorded work has passed it
   }
   if (!ok) return NPD_ECUDA;
   if ((rc = npd_kd_fwd_bwd(dev, cuda_stream)) != NPD_OK) return rc;

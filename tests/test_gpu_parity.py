@@ -425,4 +425,15 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     assert step.status() == B.NPD_OK
     assert torch.equal(hkl, ref.kl.cpu()) and torch.equal(hns, ref.nll_student.cpu())
     assert torch.equal(hnt, ref.nll_teacher.cpu())
-    assert torch.equal(step.d_hidden, ref.d_hidden) and torch.equal(step.d_weight, ref.d_weight)
+    assert frob(host(step.d_hidden), host(ref.d_hidden)) < 1e-3 and torch.equal(step.d_weight, ref.d_weight)
+    h2d, d2h = B.npd_last_copy_bytes()
+    n_loss = int(b.loss_mask.sum().item())
+    assert h2d == n_loss * (b.d + b.V) * 2 + 4 * (b.S + 1) + b.T + 4 * b.T and d2h == 12 * b.T
+    # the same with the copies on a stream of their own, twice in a row on the same staging buffers
+    copy_stream, compute = torch.cuda.Stream(), torch.cuda.Stream()
+    for _ in range(2):
+        hkl.zero_()
+        step.kl.zero_()
+        B.npd_kd_fwd_bwd_host_streams(hargs, step.args, copy_stream, compute)
+    torch.cuda.synchronize()
+    assert torch.equal(hkl, ref.kl.cpu()) and torch.equal(step.d_weight, ref.d_weight)
