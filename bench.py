@@ -354,8 +354,8 @@ def run_ours(args):
     peaks = _peaks()
     T, d, V = wl["T"], wl["d"], wl["V"]
     # Tokens without loss (the masked prompts) have zero loss and zero gradient, and the library
-    # spends no tile on the 128-row blocks that hold none.  So the work the method defines is
-    # counted on the tokens that carry loss; rows the kernels pad blocks with count as waste.
+    # computes nothing for them (it works on the compacted loss tokens).  So the work the method
+    # defines is counted on the tokens that carry loss.
     T_loss = b.n_loss
     tdv2 = 2.0 * T_loss * d * V
     # dominant kernel = the launch group with the largest share of the step

@@ -1,9 +1,9 @@
 // Fused LM-head tile kernel of the distillation step.
 //
-// For a 128-token row block and a run of 256-wide vocabulary tiles it forms the
-// student logits O_S = H W^T (Algorithm 1, "Compute Student Logits") on
-// tcgen05 tensor cores with the accumulator in tensor memory, streams the
-// matching teacher-logit tile O_T through shared memory with TMA, and consumes
+// For a block of 128 compact rows (the tokens that carry loss, numbered in packed order) and a
+// run of 256-wide vocabulary tiles it forms the student logits O_S = H W^T (Algorithm 1,
+// "Compute Student Logits") on tcgen05 tensor cores with the accumulator in tensor memory,
+// streams the matching teacher-logit tile O_T through shared memory with TMA, and consumes
 // both on chip.  The T x V logits are never written to global memory.
 //
 //   kForward : online softmax statistics of Softmax(O_T/tau) and Softmax(O_S/tau)
@@ -29,7 +29,8 @@
 //   warp 1      leader CTA (cluster rank 0) only: tcgen05.mma issuer for the pair; commits
 //               are multicast so that "stage free" and "accumulator ready" reach both CTAs.
 //               In both CTAs this warp owns the 512 TMEM columns (2 accumulators 128x256).
-//   warp 2      TMA producer for this CTA's teacher sub-tiles (two 2-stage rings)
+//   warp 2      TMA producer for this CTA's teacher sub-tiles (two 2-stage rings); the rows of a
+//               block lie anywhere in the packed batch, so each lane gathers four of them
 //   warps 4-11  epilogue; warp w reads TMEM lanes 32*(w%4).., columns 128*((w-4)/4)..
 //               so every thread owns one token row and half of the tile's columns.
 // All exponentials are taken in base 2 on logits pre-scaled by log2(e)/tau.

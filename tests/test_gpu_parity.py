@@ -230,8 +230,8 @@ def test_all_tokens_masked_gives_zero_loss_and_zero_gradients():
     [(999, 1000)],                                       # ... which is the very last row
 ])
 def test_loss_tokens_in_scattered_stretches(ranges):
-    # the kernels only visit 128-row blocks that start at loss tokens; everything else must
-    # still come out as exact zeros, and nothing may leak between blocks
+    # the kernels only compute the (compacted) loss tokens; everything else must still come out
+    # as exact zeros, and nothing may leak between neighbouring rows of a block
     b = syn.scaled("c2", device=DEV, T=1000, d=128, V=1304, seed_base=11, min_len=50, max_len=400)
     b.loss_mask[:] = 0
     for lo, hi in ranges:
