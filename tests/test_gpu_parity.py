@@ -256,6 +256,50 @@ def test_many_blocks_long_batch_small_vocabulary():
     check_full_parity(b, step)
 
 
+@pytest.mark.parametrize("seed", range(14))
+def test_random_shapes_masks_and_modes(seed):
+    # seeded random problems: odd sizes, masks from all-but-one-zero to all-one, every mode
+    rng = np.random.default_rng(100 + seed)
+    T = int(rng.integers(1, 700))
+    d = int(rng.choice([64, 128, 192]))
+    V = int(rng.integers(1, 260)) * 8
+    tau = float(rng.choice([1.0, 1.0, 0.7, 2.5]))
+    b = syn.scaled("c2", device=DEV, T=T, d=d, V=V, seed_base=300 + seed, min_len=1, max_len=max(2, T // 2))
+    b.tau = tau
+    density = float(rng.choice([0.02, 0.3, 0.7, 1.0]))
+    mask = (rng.random(T) < density).astype(np.uint8)
+    mask[int(rng.integers(0, T))] = 1
+    b.loss_mask = torch.from_numpy(mask).to(DEV)
+    mode = seed % 4
+    kw = dict(dw_dtype=torch.float32 if seed % 2 else torch.bfloat16,
+              grad_chunk_cols=int(rng.choice([0, 256, 512, 1024])))
+    H, W, Z, y, m = oracle_inputs(b)
+    if mode in (0, 1):          # dense teacher, Eq. 2 alone or the composite objective
+        lam = None if mode == 0 else float(rng.choice([0.0, 0.5, 0.9]))
+        step = run_step(b, kd_lambda=lam, **kw)
+        kl, ns, nt = orc.kd_token_losses(H, W, Z, y, m, tau)
+        assert_losses_close(host(step.nll_teacher), nt, "nll_teacher")
+        dH, dW = (orc.kd_backward(H, W, Z, m, tau, step.grad_scale) if lam is None else
+                  orc.composite_backward(H, W, Z, y, m, tau, step.grad_scale, lam))
+    else:                       # top-k teacher, with or without the cross-entropy term
+        k = int(min(V, rng.integers(1, 17)))
+        vals, idx = _topk_of(b, k)
+        lam = None if mode == 2 else 0.9
+        step = run_step(b, topk_values=vals, topk_indices=idx, kd_lambda=lam, **kw)
+        v, i = host(vals), idx.cpu().numpy()
+        kl, ns = orc.topk_kd_token_losses(H, W, v, i, y, m, tau)
+        dense = np.full_like(Z, -np.inf)
+        np.put_along_axis(dense, i.astype(np.int64), v, axis=1)
+        dH, dW = (orc.topk_kd_backward(H, W, v, i, m, tau, step.grad_scale) if lam is None else
+                  orc.composite_backward(H, W, dense, y, m, tau, step.grad_scale, lam))
+    assert_losses_close(host(step.kl), kl, "kl")
+    assert_losses_close(host(step.nll_student), ns, "nll_student")
+    if np.linalg.norm(dH) > 0:
+        assert frob(host(step.d_hidden), dH) <= GRAD_FROB
+        assert frob(host(step.d_weight), dW) <= GRAD_FROB
+    assert np.all(host(step.d_hidden)[m == 0] == 0) and np.all(host(step.kl)[m == 0] == 0)
+
+
 def test_optional_inputs_may_be_null():
     b = _mini()
     H, W, Z, y, m = oracle_inputs(b)
