@@ -208,7 +208,7 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
-def _time_e2e(B, syn, b, step, seg_out, pairs, n_pairs, stream, args, world, dev, wl):
+def _time_e2e(B, syn, b, step, seg_out, pairs, n_pairs, stream, args, world, dev, wl, topk):
     """The same step through npd_kd_fwd_bwd_host: every step copies hidden states, teacher
     logits, boundaries, mask and labels from pinned host memory and reads the per-token
     losses back, inside the timed region.  As a training loop would, the steps alternate
@@ -216,7 +216,9 @@ def _time_e2e(B, syn, b, step, seg_out, pairs, n_pairs, stream, args, world, dev
     stream, so that the copies of one step run while the kernels of the step before are still
     busy; every step's copies and kernels lie inside the timed region."""
     pin = lambda t: t.cpu().pin_memory()
-    hh, hz, hcu, hm, hy = map(pin, (b.hidden, b.teacher, b.cu_seqlens, b.loss_mask, b.labels))
+    hh, hcu, hm, hy = map(pin, (b.hidden, b.cu_seqlens, b.loss_mask, b.labels))
+    hz = None if topk else pin(b.teacher)
+    htk = {k2: pin(v) for k2, v in topk.items()}
     lanes = []
     for k in range(2):
         if k == 0:
@@ -226,12 +228,13 @@ def _time_e2e(B, syn, b, step, seg_out, pairs, n_pairs, stream, args, world, dev
                                torch.empty_like(b.teacher), torch.empty_like(b.cu_seqlens),
                                torch.empty_like(b.loss_mask), torch.empty_like(b.labels), b.tau)
             st_b.loss_mask.copy_(b.loss_mask)      # KDStep reads the loss-token count once
-            st_step = B.KDStep(st_b, grad_chunk_cols=args.grad_chunk_cols, grad_scale=step.grad_scale)
+            st_topk = {k2: torch.empty_like(v) for k2, v in topk.items()}
+            st_step = B.KDStep(st_b, grad_chunk_cols=args.grad_chunk_cols, grad_scale=step.grad_scale, **st_topk)
             st_seg = {k2: torch.empty_like(v) for k2, v in seg_out.items()}
             st_stream = torch.cuda.Stream(device=dev)
         hkl, hns, hnt = (torch.empty(b.T).pin_memory() for _ in range(3))
         hargs = B.make_kd_args(hh, b.weight, hz, cu_seqlens=hcu, loss_mask=hm, labels=hy, kl=hkl,
-                               nll_student=hns, nll_teacher=hnt, temperature=b.tau)
+                               nll_student=hns, nll_teacher=None if topk else hnt, temperature=b.tau, **htk)
         lanes.append((st_b, st_step, st_seg, st_stream, hargs, (hkl, hns, hnt)))
     steps = max(4, min(args.steps, 10))
     copy_stream = torch.cuda.Stream(device=dev)
@@ -346,8 +349,8 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry point ----
     e2e = None
-    if not args.no_e2e and args.teacher == "dense":
-        e2e = _time_e2e(B, syn, b, step, seg_out, pairs, n_pairs, stream, args, world, dev, wl)
+    if not args.no_e2e:
+        e2e = _time_e2e(B, syn, b, step, seg_out, pairs, n_pairs, stream, args, world, dev, wl, topk)
 
     if rank != 0:
         return
@@ -420,7 +423,7 @@ def main():
     ap.add_argument("--d", type=int, default=WORKLOAD["d"], help="hidden size; as for --T")
     ap.add_argument("--grad-chunk-cols", type=int, default=0, help="0 = library default")
     ap.add_argument("--teacher", default="dense", choices=["dense", "topk"],
-                    help="dense = the benchmark's workload; topk = k=10 stored logits (implies --no-e2e)")
+                    help="dense = the benchmark's workload; topk = k=10 stored logits")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
