@@ -92,10 +92,11 @@ typedef struct npd_kd_args {
   int32_t T, d, V, S;
   const void* hidden;        /* bf16 [T, ldh]   H                                  */
   const void* weight;        /* bf16 [V, ldw]   W (LM head, no bias)               */
-  const void* teacher;       /* bf16 [T, ldt]   O_T, ldt >= V; columns >= V ignored
+  const void* teacher;       /* bf16 (or f32) [T, ldt]   O_T, ldt >= V; columns >= V ignored
                                 (not read when topk > 0, see the end of the struct) */
   int64_t ldh, ldw, ldt;
-  int32_t teacher_dtype;     /* NPD_DTYPE_BF16 (NPD_DTYPE_F32: NPD_EUNSUPPORTED)    */
+  int32_t teacher_dtype;     /* NPD_DTYPE_BF16, or NPD_DTYPE_F32 (then teacher is f32
+                                [T, ldt] with ldt a multiple of 4)                   */
   int32_t reserved0;
   const int32_t* cu_seqlens; /* [S+1] cu[0]=0, strictly increasing, cu[S]=T; may be NULL
                                 (then S is ignored and nothing is validated)       */

@@ -39,6 +39,11 @@
 // of a dense row.  The forward then keeps the student's statistics only (the k teacher terms
 // are evaluated per token afterwards), warp 2 has nothing to stream, and the gradient tile is
 // coef_t p_S minus the k stored teacher probabilities at their columns.
+//
+// kTeacherF32: the dense teacher logits are fp32.  A sub-tile is then 128 rows x 32 columns
+// (again 128-byte rows, 16 KB), read without unpacking; the bf16 gradient sub-tile (64-byte
+// rows) no longer has the teacher's layout, so it is written unswizzled to the start of the
+// stage once every thread of the half has its teacher values in registers.
 #pragma once
 
 #include "ptx_sm100.cuh"
@@ -112,12 +117,13 @@ constexpr float kNegClamp = -30000.0f;
 constexpr int kMaxTopK = 16;  // stored teacher logits per token the sparse path keeps in registers
 }  // namespace kd_cfg
 
-template <int kMode, bool kTauIsOne, bool kComposite, bool kSparse>
+template <int kMode, bool kTauIsOne, bool kComposite, bool kSparse, bool kTeacherF32>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kd_cfg::THREADS, 1)
 kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant__ CUtensorMap tmap_w,
                const __grid_constant__ CUtensorMap tmap_t, const __grid_constant__ CUtensorMap tmap_g,
                const KdTileParams p) {
   using namespace kd_cfg;
+  constexpr int ZC = kTeacherF32 ? 32 : ZSUB_COLS;  // columns of a teacher sub-tile (128-byte rows)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~static_cast<uintptr_t>(1023));
@@ -260,10 +266,10 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
 #pragma unroll
         for (int i = 0; i < 4; ++i) tr[i] = r < 0 ? 0 : __ldg(p.rows + r + 4 * lane + i);
         for (int vt = vt0; vt < vt1 && ok; ++vt) {
-          for (int j = 0; j < BN / 2 / ZSUB_COLS && ok; ++j, ++zit) {
+          for (int j = 0; j < BN / 2 / ZC && ok; ++j, ++zit) {
             const uint32_t q = zit % ZQ, ph = (zit / ZQ) & 1;
             for (int half = 0; half < 2; ++half) {
-              const int col = vt * BN + half * (BN / 2) + j * ZSUB_COLS;
+              const int col = vt * BN + half * (BN / 2) + j * ZC;
               const uint32_t bi = 8 * (half * ZQ + q);
               ok = __all_sync(0xffffffffu, mbar_wait(zempty0 + bi, ph ^ 1, abort_flag));
               if (!ok) break;
@@ -330,7 +336,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         tc_fence_after_sync();
         const uint32_t taddr =
             tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN + half * (BN / 2);
-        for (int j = 0; j < BN / 2 / ZSUB_COLS && ok; ++j, ++zit) {
+        for (int j = 0; j < BN / 2 / ZC && ok; ++j, ++zit) {
           const uint32_t q = zit % ZQ, zph = (zit / ZQ) & 1;
           const uint32_t bi = 8 * (half * ZQ + q);
           if (!kSparse) {
@@ -338,29 +344,35 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
             if (!ok) break;
           }
           uint8_t* zrow = smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES + row_local * 128;
-          const int sub_col0 = vt * BN + half * (BN / 2) + j * ZSUB_COLS;
+          const int sub_col0 = vt * BN + half * (BN / 2) + j * ZC;
 #pragma unroll 1
-          for (int c = 0; c < ZSUB_COLS / 32; ++c) {
+          for (int c = 0; c < ZC / 32; ++c) {
             const int col0 = sub_col0 + c * 32;
             uint32_t acc[32];
-            tmem_ld32(taddr + j * ZSUB_COLS + c * 32, acc);
-            uint4 zq[4];
+            tmem_ld32(taddr + j * ZC + c * 32, acc);
+            constexpr int NZQ = kTeacherF32 ? 8 : 4;  // 16-byte pieces that hold this chunk's 32 logits
+            uint4 zq[NZQ];
             if (!kSparse) {
 #pragma unroll
-              for (int i = 0; i < 4; ++i)
-                zq[i] = *reinterpret_cast<const uint4*>(zrow + ((static_cast<uint32_t>(c * 4 + i) ^ swz) << 4));
+              for (int i = 0; i < NZQ; ++i)
+                zq[i] = *reinterpret_cast<const uint4*>(
+                    zrow + ((static_cast<uint32_t>(kTeacherF32 ? i : c * 4 + i) ^ swz) << 4));
             }
             tmem_ld_wait();
             const int nvalid = p.V - col0;  // columns of this chunk inside the vocabulary
             float zt[32];
             if (!kSparse) {
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
+              for (int i = 0; i < NZQ; ++i) {
                 const uint32_t w[4] = {zq[i].x, zq[i].y, zq[i].z, zq[i].w};
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                  zt[8 * i + 2 * k] = fmaxf(bf16_lo(w[k]), kNegClamp);
-                  zt[8 * i + 2 * k + 1] = fmaxf(bf16_hi(w[k]), kNegClamp);
+                  if (kTeacherF32) {
+                    zt[4 * i + k] = fmaxf(__uint_as_float(w[k]), kNegClamp);
+                  } else {
+                    zt[8 * i + 2 * k] = fmaxf(bf16_lo(w[k]), kNegClamp);
+                    zt[8 * i + 2 * k + 1] = fmaxf(bf16_hi(w[k]), kNegClamp);
+                  }
                 }
               }
             }
@@ -460,10 +472,21 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
 #pragma unroll
               for (int i = 0; i < 32; i += 2)
                 packed[i >> 1] = pack_bf16x2(i < nvalid ? g[i] : 0.f, i + 1 < nvalid ? g[i + 1] : 0.f);
+              if (kTeacherF32) {
+                // 64-byte gradient rows, dense from the start of the stage: they overlap other
+                // threads' teacher rows, so everyone of this half must have read its row first
+                named_barrier_sync(1 + half, 128);
+                uint8_t* grow = smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES + row_local * 64;
 #pragma unroll
-              for (int i = 0; i < 4; ++i)
-                *reinterpret_cast<uint4*>(zrow + ((static_cast<uint32_t>(c * 4 + i) ^ swz) << 4)) =
-                    make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+                for (int i = 0; i < 4; ++i)
+                  *reinterpret_cast<uint4*>(grow + 16 * i) =
+                      make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                  *reinterpret_cast<uint4*>(zrow + ((static_cast<uint32_t>(c * 4 + i) ^ swz) << 4)) =
+                      make_uint4(packed[4 * i], packed[4 * i + 1], packed[4 * i + 2], packed[4 * i + 3]);
+              }
             }
           }
           if (kMode == kForward) {

@@ -43,7 +43,7 @@ PFN_cuTensorMapEncodeTiled_v12000 tensor_map_encoder() {
 // 2-D tensor map with 128-byte swizzle.  inner = contiguous extent (elements), outer = rows,
 // ld = row stride (elements), box = {box_inner (128 bytes' worth), box_outer}.
 bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t ld,
-              uint32_t box_inner, uint32_t box_outer, bool f32 = false) {
+              uint32_t box_inner, uint32_t box_outer, bool f32 = false, bool swizzle = true) {
   auto enc = tensor_map_encoder();
   if (enc == nullptr) return false;
   cuuint64_t dims[2] = {inner, outer};
@@ -52,7 +52,8 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, 
   cuuint32_t estr[2] = {1, 1};
   return enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
              const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+             CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -146,8 +147,8 @@ int check_args(const npd_kd_args* a, bool need_pointers) {
   if (a == nullptr || a->size != sizeof(npd_kd_args)) return NPD_EINVAL;
   if (a->T < 1 || a->d < 1 || a->V < 1) return NPD_EINVAL;
   if (!(a->temperature > 0.f) || !std::isfinite(a->temperature)) return NPD_EINVAL;
-  if (a->teacher_dtype == NPD_DTYPE_F32) return NPD_EUNSUPPORTED;
-  if (a->teacher_dtype != NPD_DTYPE_BF16) return NPD_EINVAL;
+  if (a->teacher_dtype != NPD_DTYPE_BF16 && a->teacher_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
+  const bool tf32 = a->teacher_dtype == NPD_DTYPE_F32;
   if (a->d_weight_dtype != NPD_DTYPE_BF16 && a->d_weight_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
   if (a->grad_chunk_cols < 0 || a->n_phase_events < 0) return NPD_EINVAL;
   if (a->d % 64 != 0) return NPD_ESHAPE;
@@ -156,7 +157,7 @@ int check_args(const npd_kd_args* a, bool need_pointers) {
   if (sparse && a->topk > kd_cfg::kMaxTopK) return NPD_EUNSUPPORTED;
   if (a->ldh < a->d || a->ldw < a->d || (!sparse && a->ldt < a->V)) return NPD_ESHAPE;
   if (a->cu_seqlens != nullptr && (a->S < 1 || a->S > a->T)) return NPD_ESHAPE;
-  if ((a->ldh % 8) || (a->ldw % 8) || (!sparse && (a->ldt % 8))) return NPD_EALIGN;
+  if ((a->ldh % 8) || (a->ldw % 8) || (!sparse && (a->ldt % (tf32 ? 4 : 8)))) return NPD_EALIGN;
   if ((a->d_hidden == nullptr) != (a->d_weight == nullptr)) return NPD_EINVAL;
   if ((a->flags & NPD_KD_ACCUMULATE_DW) && a->d_weight_dtype != NPD_DTYPE_F32) return NPD_EINVAL;
   if ((a->flags & NPD_KD_REVERSE_KL) && (a->d_hidden != nullptr || a->topk != 0)) return NPD_EINVAL;
@@ -240,17 +241,20 @@ int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const
 }
 
 template <int kMode>
-int launch_kd_tile(bool tau_one, bool composite, bool sparse, const CUtensorMap& mh, const CUtensorMap& mw, const CUtensorMap& mt,
+int launch_kd_tile(bool tau_one, bool composite, bool sparse, bool tf32, const CUtensorMap& mh, const CUtensorMap& mw, const CUtensorMap& mt,
                    const CUtensorMap& mg, const KdTileParams& kp, int sms, cudaStream_t st) {
   using namespace kd_cfg;
   composite = composite && kMode == kGradient;  // the forward does not depend on the objective's mix
-  auto k = kd_tile_kernel<kMode, true, false, false>;
-  if (!sparse) {
-    if (!composite) k = tau_one ? kd_tile_kernel<kMode, true, false, false> : kd_tile_kernel<kMode, false, false, false>;
-    else k = tau_one ? kd_tile_kernel<kMode, true, true, false> : kd_tile_kernel<kMode, false, true, false>;
+  auto k = kd_tile_kernel<kMode, true, false, false, false>;
+  if (sparse) {
+    if (!composite) k = tau_one ? kd_tile_kernel<kMode, true, false, true, false> : kd_tile_kernel<kMode, false, false, true, false>;
+    else k = tau_one ? kd_tile_kernel<kMode, true, true, true, false> : kd_tile_kernel<kMode, false, true, true, false>;
+  } else if (tf32) {
+    if (!composite) k = tau_one ? kd_tile_kernel<kMode, true, false, false, true> : kd_tile_kernel<kMode, false, false, false, true>;
+    else k = tau_one ? kd_tile_kernel<kMode, true, true, false, true> : kd_tile_kernel<kMode, false, true, false, true>;
   } else {
-    if (!composite) k = tau_one ? kd_tile_kernel<kMode, true, false, true> : kd_tile_kernel<kMode, false, false, true>;
-    else k = tau_one ? kd_tile_kernel<kMode, true, true, true> : kd_tile_kernel<kMode, false, true, true>;
+    if (!composite) k = tau_one ? kd_tile_kernel<kMode, true, false, false, false> : kd_tile_kernel<kMode, false, false, false, false>;
+    else k = tau_one ? kd_tile_kernel<kMode, true, true, false, false> : kd_tile_kernel<kMode, false, true, false, false>;
   }
   if (set_smem(k, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
   // the number of units is only known on the device: always one CTA pair per two SMs
@@ -335,6 +339,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   const float scale2 = 1.4426950408889634f / a->temperature;
 
   const bool sparse = a->topk > 0;  // teacher stored as its top-k logits per token
+  const bool tf32 = !sparse && a->teacher_dtype == NPD_DTYPE_F32;
   float* tk_cp = reinterpret_cast<float*>(ws + pl.off_tkcp);
   CUtensorMap mh, mw, mt;
   // H is read as its compact copy; the teacher by four-row gathers (box one row high)
@@ -343,7 +348,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     return NPD_ECUDA;
   if (sparse) {
     mt = mh;  // never used: no teacher tiles are streamed
-  } else if (!make_map(&mt, a->teacher, a->V, a->T, a->ldt, 64, 1)) {
+  } else if (!make_map(&mt, a->teacher, a->V, a->T, a->ldt, tf32 ? 32 : 64, 1, tf32)) {
     return NPD_ECUDA;
   }
 
@@ -381,7 +386,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   kp.partials = partials;
   kp.reverse = (a->flags & NPD_KD_REVERSE_KL) ? 1 : 0;
   kp.status = status;
-  if ((rc = launch_kd_tile<kForward>(tau_one, false, sparse, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
+  if ((rc = launch_kd_tile<kForward>(tau_one, false, sparse, tf32, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
   rec.mark();
 
   if (sparse) {
@@ -426,7 +431,8 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   cp.partials = partials;
   cp.hidden = static_cast<const __nv_bfloat16*>(a->hidden);
   cp.weight = static_cast<const __nv_bfloat16*>(a->weight);
-  cp.teacher = static_cast<const __nv_bfloat16*>(a->teacher);
+  cp.teacher = a->teacher;
+  cp.teacher_f32 = tf32 ? 1 : 0;
   cp.ldh = a->ldh;
   cp.ldw = a->ldw;
   cp.ldt = a->ldt;
@@ -468,7 +474,9 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     if (cols <= 0) break;
     const int cols_pad = std::min(pl.chunk_cols, pl.vtiles * 256 - col0);
     CUtensorMap mg;
-    if (!make_map(&mg, gbuf, cols_pad, crows, ldg, 64, 128))
+    // gradient sub-tiles: 64 columns in the teacher's swizzled layout, or (fp32 teacher) 32 plain
+    if (!(tf32 ? make_map(&mg, gbuf, cols_pad, crows, ldg, 32, 128, false, false)
+               : make_map(&mg, gbuf, cols_pad, crows, ldg, 64, 128)))
       return NPD_ECUDA;
     KdTileParams gp = kp;
     gp.vt_begin = col0 / 256;
@@ -484,7 +492,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     gp.tk_cp = tk_cp;
     gp.topk = a->topk;
     gp.g_col0 = col0;
-    if ((rc = launch_kd_tile<kGradient>(tau_one, composite, sparse, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
+    if ((rc = launch_kd_tile<kGradient>(tau_one, composite, sparse, tf32, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
     rec.mark();
 
     GemmProblem pr[2] = {};
@@ -612,7 +620,8 @@ int npd_kd_fwd_bwd_host_streams(const npd_kd_args* host, const npd_kd_args* dev,
     copy_rows(dev->topk_indices, dev->topk, host->topk_indices, dev->topk, sizeof(int32_t) * dev->topk,
               sizeof(int32_t));
   } else {
-    copy_rows(dev->teacher, dev->ldt, host->teacher, host->ldt, static_cast<size_t>(dev->V) * 2, 2);
+    const size_t te = dev->teacher_dtype == NPD_DTYPE_F32 ? 4 : 2;
+    copy_rows(dev->teacher, dev->ldt, host->teacher, host->ldt, static_cast<size_t>(dev->V) * te, te);
   }
   if (dev->cu_seqlens != nullptr && host->cu_seqlens != nullptr) {
     ok &= cudaMemcpyAsync(const_cast<int32_t*>(dev->cu_seqlens), host->cu_seqlens,

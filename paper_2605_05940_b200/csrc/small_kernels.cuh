@@ -121,7 +121,8 @@ struct CombineParams {
   const float* partials;  // [nslots][kPFields][T]
   const __nv_bfloat16* hidden;
   const __nv_bfloat16* weight;
-  const __nv_bfloat16* teacher;
+  const void* teacher;    // bf16, or fp32 when teacher_f32
+  int teacher_f32;
   long long ldh, ldw, ldt;
   const uint8_t* loss_mask;
   const int32_t* labels;
@@ -215,7 +216,9 @@ __global__ void __launch_bounds__(256) kd_combine_kernel(const CombineParams p) 
         dot = fmaf(bf16_hi(h.w), bf16_hi(w.w), dot);
       }
       dot = warp_sum(dot);
-      const float zt_y = __bfloat162float(p.teacher[static_cast<size_t>(t) * p.ldt + y]);
+      const size_t at = static_cast<size_t>(t) * p.ldt + y;
+      const float zt_y = p.teacher_f32 ? static_cast<const float*>(p.teacher)[at]
+                                       : __bfloat162float(static_cast<const __nv_bfloat16*>(p.teacher)[at]);
       // natural-log lse of the untempered logits
       const float nat_b = kTauIsOne ? kLn2 * lse_b : kLn2 * (mb * p.tau + log2f(sb1));
       const float nat_a = kTauIsOne ? kLn2 * lse_a : kLn2 * (ma * p.tau + log2f(sa1));

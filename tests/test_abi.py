@@ -97,7 +97,9 @@ def test_argument_errors_are_found_on_the_host():
     assert _ws_rc(bad) == B.NPD_ESHAPE
     bad = B.npd_kd_args.from_buffer_copy(a); bad.ldt = 42
     assert _ws_rc(bad) == B.NPD_EALIGN
-    bad = B.npd_kd_args.from_buffer_copy(a); bad.teacher_dtype = B.NPD_DTYPE_F32
+    bad = B.npd_kd_args.from_buffer_copy(a); bad.teacher_dtype = 5
+    assert _ws_rc(bad) == B.NPD_EINVAL
+    bad = B.npd_kd_args.from_buffer_copy(a); bad.topk = 17                  # more than the kernels keep per token
     assert _ws_rc(bad) == B.NPD_EUNSUPPORTED
     bad = B.npd_kd_args.from_buffer_copy(a); bad.d_hidden = 4096            # dH without dW
     assert _ws_rc(bad) == B.NPD_EINVAL

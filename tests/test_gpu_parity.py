@@ -72,6 +72,34 @@ def test_config1_tiny_all_outputs():
     assert np.array_equal(b.cu_seqlens.cpu().numpy(), [0, 32, 96, 192, 256])
 
 
+def test_config1_tiny_with_its_fp32_teacher():
+    # the tiny configuration as stated: dense fp32 teacher logits (H and W rounded to bf16)
+    b = syn.config1_tiny(device=DEV, teacher_dtype=torch.float32)
+    assert b.teacher.dtype == torch.float32
+    step = run_step(b, dw_dtype=torch.float32)
+    assert step.args.teacher_dtype == B.NPD_DTYPE_F32
+    kl, ns, nt = check_full_parity(b, step)
+    check_stats_and_select(b, step, kl, ns, nt)
+
+
+@pytest.mark.parametrize("tau,lam,chunk", [(1.0, None, 0), (2.0, None, 512), (1.0, 0.9, 1024), (0.7, 0.5, 256)])
+def test_fp32_teacher_ragged_shapes(tau, lam, chunk):
+    b = syn.scaled("c2", device=DEV, T=700, d=128, V=3000, min_len=20, max_len=300)
+    b.tau = tau
+    g = torch.Generator(device=DEV).manual_seed(17)
+    b.teacher = b.teacher.float() + 1e-3 * torch.randn(b.teacher.shape, device=DEV, generator=g)  # not bf16-representable
+    step = run_step(b, kd_lambda=lam, grad_chunk_cols=chunk, dw_dtype=torch.float32)
+    H, W, Z, y, m = oracle_inputs(b)
+    kl, ns, nt = orc.kd_token_losses(H, W, Z, y, m, tau)
+    assert_losses_close(host(step.kl), kl, "kl")
+    assert_losses_close(host(step.nll_student), ns, "nll_student")
+    assert_losses_close(host(step.nll_teacher), nt, "nll_teacher")
+    dH, dW = (orc.kd_backward(H, W, Z, m, tau, step.grad_scale) if lam is None else
+              orc.composite_backward(H, W, Z, y, m, tau, step.grad_scale, lam))
+    assert frob(host(step.d_hidden), dH) <= GRAD_FROB and frob(host(step.d_weight), dW) <= GRAD_FROB
+    assert np.all(host(step.d_hidden)[m == 0] == 0)
+
+
 @pytest.mark.parametrize("chunk", [0, 256, 1024])
 def test_scaled_config2_multi_tile_ragged(chunk):
     # 6 row blocks with a ragged last one, 12 vocabulary tiles with a ragged tail, 2 k-steps
@@ -385,8 +413,8 @@ def test_workspace_and_option_errors():
     a.workspace = step.args.workspace + 16
     assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EWORKSPACE
     a = B.npd_kd_args.from_buffer_copy(step.args)
-    a.teacher_dtype = B.NPD_DTYPE_F32
-    assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EUNSUPPORTED
+    a.teacher_dtype = 7
+    assert B.lib().npd_kd_fwd_bwd(C.byref(a), None) == B.NPD_EINVAL
 
 
 def test_select_matches_float32_oracle_bit_for_bit():
