@@ -22,6 +22,13 @@
  *   IFD = L(A|Q)/L(A) (Eq. 3), Delta = IFD_T - IFD_S (Eq. 4),
  *   keep = lo <= Delta <= hi (Proximal Learning Zone, Section 3.2)
  *
+ * Options: the composite objective of Eq. 1 (cross-entropy term added to the gradient,
+ * NPD_KD_COMPOSITE_LOSS), the teacher stored as its k largest logits per token (Eq. 2 as
+ * printed, topk_values / topk_indices), fp32 teacher logits, the learner-to-generator KL
+ * of the policy-lag analysis (NPD_KD_REVERSE_KL), the selection scopes of the filter
+ * ablation (flags of npd_select), and the sequence packer of Algorithm 1
+ * (npd_pack_sequences).
+ *
  * Conventions
  *   - Every pointer is a DEVICE pointer unless the comment says HOST.
  *   - The caller owns every buffer.  The library allocates no device memory,
