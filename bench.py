@@ -324,17 +324,26 @@ def run_ours(args):
         assert step.status(stream) == B.NPD_OK
 
         # ---- timed region: K steps, device-timed on the launching stream ----
-        _barrier(world)
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with ClockSampler(local) as clk:
-            e0.record(stream)
-            for _ in range(args.steps):
-                one_step()
-            e1.record(stream)
-            stream.synchronize()
-        torch.cuda.synchronize()
-        _barrier(world)
+        # A run during which the GPU reported a hardware or thermal slowdown is taken again, once.
+        remeasured = False
+        for attempt in range(2):
+            _barrier(world)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with ClockSampler(local) as clk:
+                e0.record(stream)
+                for _ in range(args.steps):
+                    one_step()
+                e1.record(stream)
+                stream.synchronize()
+            torch.cuda.synchronize()
+            _barrier(world)
+            bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(clk.summary()["reasons"])
+            bad_any = _max_over_ranks(1.0 if bad else 0.0, world, dev) > 0
+            if not bad_any or attempt == 1:
+                break
+            remeasured = True
+            time.sleep(5.0)
         ms_total = _max_over_ranks(e0.elapsed_time(e1), world, dev)
         ms_step = ms_total / args.steps
         tokens_per_s = world * wl["T"] / (ms_step * 1e-3)
@@ -383,7 +392,7 @@ def run_ours(args):
                    "loss_tokens": T_loss, "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (teacher logits 2.49 GB per step)",
                    "grad_chunks": chunks, "teacher": args.teacher},
-        "clocks": clk.summary(),
+        "clocks": dict(clk.summary(), remeasured_after_slowdown=remeasured),
         "gpu_launches": launches_per_step * args.steps,
         "e2e": e2e,
         "roofline": {"bound": "tensor", "kernel": dom, "achieved": achieved, "peak": peak_tf,
