@@ -101,6 +101,21 @@ def test_config2_full_size_top_k_teacher_sampled_rows():
     assert bool(torch.isfinite(step.d_weight.float()).all())
 
 
+def test_config2_full_size_fp32_teacher_sampled_rows():
+    b = syn.config2_1b(device=DEV)
+    g = torch.Generator(device=DEV).manual_seed(23)
+    for r0 in range(0, b.T, 1024):       # fp32 logits that bf16 cannot represent, built in row slabs
+        if r0 == 0:
+            t32 = torch.empty(b.teacher.shape, dtype=torch.float32, device=DEV)
+        sl = slice(r0, min(b.T, r0 + 1024))
+        t32[sl] = b.teacher[sl].float() + 2e-3 * torch.randn((sl.stop - sl.start, b.V), device=DEV, generator=g)
+    b.teacher = t32
+    step = run_step(b)
+    assert step.args.teacher_dtype == B.NPD_DTYPE_F32
+    _check_sampled_rows(b, step, _sample_rows(b, 24, 7))
+    _check_properties(b, step)
+
+
 def test_config3_full_size_sampled_rows_temperature_two():
     b = syn.config3_rows(device=DEV)
     assert (b.T, b.d, b.tau) == (32768, 2048, 2.0)
