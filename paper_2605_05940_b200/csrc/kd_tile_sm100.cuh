@@ -24,12 +24,12 @@
 // the logits of its own 128 tokens for all 256 columns.
 //
 // CTA = 384 threads, one CTA per SM, persistent over work units:
-//   warp 0      TMA producer for this CTA's H and W operand stages (5-stage ring); the
+//   warp 0      TMA producer for this CTA's H and W operand stages (4- or 5-stage ring); the
 //               completion of both CTAs' loads is counted on the leader's "full" barrier
 //   warp 1      leader CTA (cluster rank 0) only: tcgen05.mma issuer for the pair; commits
 //               are multicast so that "stage free" and "accumulator ready" reach both CTAs.
 //               In both CTAs this warp owns the 512 TMEM columns (2 accumulators 128x256).
-//   warp 2      TMA producer for this CTA's teacher sub-tiles (two 2-stage rings); the rows of a
+//   warp 2      TMA producer for this CTA's teacher sub-tiles (a ring of 2 or 3 stages per column half); the rows of a
 //               block lie anywhere in the packed batch, so each lane gathers four of them
 //   warps 4-11  epilogue; warp w reads TMEM lanes 32*(w%4).., columns 128*((w-4)/4)..
 //               so every thread owns one token row and half of the tile's columns.
@@ -95,20 +95,28 @@ struct KdTileParams {
 namespace kd_cfg {
 constexpr int BM = 128, BN = 256, BK = 64, UK = 16;  // BM = token rows per CTA (256 per pair)
 constexpr int BNH = BN / 2;                // weight rows each CTA of the pair stages
-constexpr int STAGES = 5;
 constexpr int A_BYTES = BM * BK * 2;       // 16 KB
 constexpr int B_BYTES = BNH * BK * 2;      // 16 KB
 constexpr int ZSUB_COLS = 64;              // teacher sub-tile: 128 rows x 64 bf16 (128 B rows)
 constexpr int ZSUB_BYTES = BM * ZSUB_COLS * 2;  // 16 KB
-constexpr int ZQ = 2;                      // ring depth per column half
 constexpr int THREADS = 384;
 constexpr int TMEM_COLS = 512;
-constexpr int OFF_A = 0;
-constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-constexpr int OFF_Z = OFF_B + STAGES * B_BYTES;
-constexpr int OFF_BAR = OFF_Z + 2 * ZQ * ZSUB_BYTES;
-constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * ZQ;
-constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;
+// Shared-memory layout.  224 KB go to the operand ring (32 KB per stage) and to the teacher
+// stages (16 KB each, per column half).  Both kernels are bound by the operand feed from L2,
+// not by its latency, so ring depth beyond four buys nothing; the forward pass puts the spare
+// 32 KB into a third teacher stage per half (measured: 1.3 % faster), the gradient pass, whose
+// teacher stages double as staging for the gradient tiles, is faster with 5 + 2.
+template <int kMode>
+struct Layout {
+  static constexpr int STAGES = kMode == 0 ? 4 : 5;  // operand ring depth
+  static constexpr int ZQ = kMode == 0 ? 3 : 2;      // teacher ring depth per column half
+  static constexpr int OFF_A = 0;
+  static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
+  static constexpr int OFF_Z = OFF_B + STAGES * B_BYTES;
+  static constexpr int OFF_BAR = OFF_Z + 2 * ZQ * ZSUB_BYTES;
+  static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * ZQ;
+  static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;
+};
 // Teacher logits are clamped below at this value: a finite stand-in for the -inf entries of
 // a densified top-k teacher.  It is small enough that 2^((clamp - row max) * scale) is 0 for
 // any sane row, and small enough in magnitude that fp32 still resolves differences of scaled
@@ -123,6 +131,9 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                const __grid_constant__ CUtensorMap tmap_t, const __grid_constant__ CUtensorMap tmap_g,
                const KdTileParams p) {
   using namespace kd_cfg;
+  using L = Layout<kMode>;
+  constexpr int STAGES = L::STAGES, ZQ = L::ZQ, OFF_A = L::OFF_A, OFF_B = L::OFF_B, OFF_Z = L::OFF_Z,
+                OFF_BAR = L::OFF_BAR, NUM_BARS = L::NUM_BARS;
   constexpr int ZC = kTeacherF32 ? 32 : ZSUB_COLS;  // columns of a teacher sub-tile (128-byte rows)
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &

@@ -256,10 +256,10 @@ int launch_kd_tile(bool tau_one, bool composite, bool sparse, bool tf32, const C
     if (!composite) k = tau_one ? kd_tile_kernel<kMode, true, false, false, false> : kd_tile_kernel<kMode, false, false, false, false>;
     else k = tau_one ? kd_tile_kernel<kMode, true, true, false, false> : kd_tile_kernel<kMode, false, true, false, false>;
   }
-  if (set_smem(k, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
+  if (set_smem(k, Layout<kMode>::SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
   // the number of units is only known on the device: always one CTA pair per two SMs
   const int grid = 2 * std::max(sms / 2, 1);
-  k<<<grid, THREADS, SMEM_BYTES, st>>>(mh, mw, mt, mg, kp);
+  k<<<grid, THREADS, Layout<kMode>::SMEM_BYTES, st>>>(mh, mw, mt, mg, kp);
   ++g_launches;
   return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
 }
