@@ -283,7 +283,10 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     from paper_2605_05940_b200 import binding as B, build as npd_build, synth_inputs as syn
-    npd_build.build()
+    # one rank per node (re)builds the library if it is stale; the others wait for it
+    if local == 0:
+        npd_build.build()
+    _barrier(world)
 
     wl = dict(WORKLOAD, T=args.T, d=args.d)
     # every rank draws its own batch (independent replicas)
