@@ -167,6 +167,10 @@ int npd_phase_count(const npd_kd_args* args, int32_t* out_groups, int32_t* out_c
  * on the rest, so a batch with 30 % masked prompt tokens costs 30 % less.  Every output
  * element is written all the same (zeros where nothing is computed).
  *
+ * The call makes no synchronising CUDA call; it can be recorded by a stream capture and
+ * replayed as a CUDA graph (the tensor maps in the launch arguments bake in the buffer
+ * addresses of the captured call).
+ *
  * kl, nll_*, and d_weight are bitwise reproducible from run to run.  d_hidden is summed
  * over vocabulary chunks with fp32 atomic adds whose order is not fixed: a few of its
  * bf16 elements may round differently between runs. */

@@ -328,6 +328,27 @@ def test_random_shapes_masks_and_modes(seed):
     assert np.all(host(step.d_hidden)[m == 0] == 0) and np.all(host(step.kl)[m == 0] == 0)
 
 
+def test_step_can_be_captured_in_a_cuda_graph_and_replayed():
+    # the whole step only enqueues work on the given stream, so a stream capture records it
+    b = syn.scaled("c2", device=DEV, T=700, d=128, V=3000, min_len=20, max_len=300)
+    step = run_step(b, dw_dtype=torch.float32, grad_chunk_cols=1024)     # eager, also warms everything up
+    want = [t.clone() for t in (step.kl, step.nll_student, step.nll_teacher, step.d_weight)]
+    dh = step.d_hidden.clone()
+    s = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.graph(g, stream=s):
+        step.run(torch.cuda.current_stream())
+    for t in (step.kl, step.nll_student, step.nll_teacher, step.d_weight, step.d_hidden):
+        t.fill_(float("nan"))
+    g.replay()
+    torch.cuda.synchronize()
+    assert step.status() == B.NPD_OK
+    for w, t in zip(want, (step.kl, step.nll_student, step.nll_teacher, step.d_weight)):
+        assert torch.equal(w, t)
+    assert frob(host(step.d_hidden), host(dh)) < 1e-3
+
+
 def test_optional_inputs_may_be_null():
     b = _mini()
     H, W, Z, y, m = oracle_inputs(b)
