@@ -67,6 +67,13 @@ def lib() -> C.CDLL:
     """The loaded library.  Raises if it has not been built (no fallback)."""
     global _lib
     if _lib is None:
+        from . import build as _build
+        if _build.is_stale():          # missing, or built from other sources than the ones present
+            try:
+                _build.build()
+            except RuntimeError:
+                if not os.path.exists(LIB_PATH):
+                    raise
         if not os.path.exists(LIB_PATH):
             raise RuntimeError(
                 f"{LIB_PATH} is missing: build it with `python -m paper_2605_05940_b200.build` "

@@ -2,6 +2,7 @@
 
 from __future__ import annotations
 
+import hashlib
 import os
 import shutil
 import subprocess
@@ -22,11 +23,24 @@ def nvcc_path() -> str:
     return cand
 
 
+STAMP_PATH = LIB_PATH + ".sources"   # digest of the sources the library was built from
+
+
+def sources_digest() -> str:
+    h = hashlib.sha256()
+    for d in sorted(DEPS):
+        with open(d, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+    """True when there is no library or it was built from other sources (by content, not by
+    time stamps: a copied tree does not keep them in order)."""
+    if not (os.path.exists(LIB_PATH) and os.path.exists(STAMP_PATH)):
         return True
-    t = os.path.getmtime(LIB_PATH)
-    return any(os.path.getmtime(d) > t for d in DEPS)
+    with open(STAMP_PATH) as f:
+        return f.read().strip() != sources_digest()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -43,6 +57,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         sys.stderr.write(res.stderr)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    with open(STAMP_PATH, "w") as f:
+        f.write(sources_digest() + "\n")
     return LIB_PATH
 
 
