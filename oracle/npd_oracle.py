@@ -64,6 +64,7 @@ __all__ = [
     "reverse_kl_token",
     "ifd_scores",
     "delta_ifd_select",
+    "perplexity_scores",
     "nearest_rank_percentile",
     "pack_first_fit_decreasing",
 ]
@@ -425,6 +426,29 @@ def delta_ifd_select(cond_seg, uncond_seg, nll_s_sum, nll_t_sum, count,
             keep &= ifd_t <= f(1.0)
     keep &= ~np.isnan(tested)
     return ifd_t, ifd_s, delta, keep.astype(np.uint8), int(keep.sum())
+
+
+def perplexity_scores(seg, nll_sum, count, dtype=np.float64):
+    """Per-sample perplexity, the classical filtering metric of the filter ablation (table of
+    filtering metrics, row "Perplexity (PPL)"):
+
+        PPL_i = exp( nll_sum[seg_i] / count[seg_i] ),
+
+    the exponential of the token-mean cross-entropy of the sample's answer tokens (the same
+    per-sequence loss L_theta that Eq. 3 divides), i.e. the inverse geometric mean of the
+    probabilities the model gives the answer tokens.  A sample without such tokens scores NaN.
+    The paper lists the metric with the scope "Weighted" and does not say how the weight enters
+    training, so only the score is defined here.  ``dtype`` is the arithmetic type of the two
+    operations (one mean, one exponential)."""
+    f = np.dtype(dtype).type
+    si = np.asarray(seg, dtype=np.int64)
+    nll_sum = np.asarray(nll_sum).astype(dtype)
+    count = np.asarray(count)
+    out = np.empty(si.size, dtype=dtype)
+    for i in range(si.size):
+        n = int(count[si[i]])
+        out[i] = np.exp(f(nll_sum[si[i]]) / f(n)) if n > 0 else np.nan
+    return out
 
 
 def nearest_rank_percentile(values, q: float) -> float:

@@ -3,7 +3,17 @@ run the oracle on the same inputs, compare with the stated tolerances.
 
 Tolerances (bf16 operands, fp32 accumulation and softmax; bf16 gradient tiles):
   per-token losses   |gpu - ref| <= 2e-3 * |ref| + 1e-6
-  gradients          ||gpu - ref||_F / ||ref||_F <= 1e-2   (bf16 gradient tiles)
+  gradients          ||gpu - ref||_F / ||ref||_F <= 1e-2   (bf16 gradient tiles), over the whole
+                     matrix AND, at 2e-2, over every block of 128 rows of dH and of 256 rows of dW
+                     (the row extents of the kernels' tiles), so that one wrong tile, stripe or
+                     chunk offset cannot hide in the norm of a large matrix.  Why 2e-2: an element
+                     of a gradient is a sum of products whose logit-gradient factor was rounded to
+                     bf16 (relative error <= 2^-9, about 1.1e-3 rms) and the result is rounded to
+                     bf16 once more; both errors are independent per element, so the relative
+                     Frobenius error of any block is about 2e-3 whatever its size.  The block bound
+                     keeps the same factor of ~5-10 of slack over that as the matrix bound does.
+                     Blocks whose reference norm is below 1e-3 of the mean block norm are skipped
+                     (their entries are rounding noise of the larger rows' scale).
   counts, segment ids, cu boundaries   bit-exact
   keep mask          bit-exact except samples whose Delta lies within 1e-4 of lo or hi
 """
@@ -16,6 +26,7 @@ from paper_2605_05940_b200 import binding as B
 
 LOSS_RTOL, LOSS_ATOL = 2e-3, 1e-6
 GRAD_FROB = 1e-2
+GRAD_FROB_BLOCK = 2e-2
 BAND = 1e-4
 
 
@@ -25,6 +36,89 @@ def host(t):
 
 def frob(a, r):
     return float(np.linalg.norm(np.asarray(a, np.float64) - r) / max(np.linalg.norm(r), 1e-300))
+
+
+def assert_blocks_close(got, ref, block_rows, what):
+    """Relative Frobenius error of every block of `block_rows` consecutive rows."""
+    got, ref = np.asarray(got, np.float64), np.asarray(ref, np.float64)
+    n = -(-ref.shape[0] // block_rows)
+    pad = n * block_rows - ref.shape[0]
+    sq = lambda a: np.add.reduceat((a * a).sum(axis=1), np.arange(0, a.shape[0], block_rows))
+    err, nrm = np.sqrt(sq(got - ref)), np.sqrt(sq(ref))
+    floor = 1e-3 * np.sqrt(np.mean(nrm ** 2))
+    live = nrm > floor
+    bad = live & (err > GRAD_FROB_BLOCK * nrm)
+    # a block that should be (almost) zero must be (almost) zero
+    bad |= ~live & (err > GRAD_FROB_BLOCK * max(floor, 1e-300))
+    assert not bad.any(), f"{what}: blocks {np.flatnonzero(bad)[:8]} of {n} ({block_rows} rows each, " \
+                          f"last one {block_rows - pad}) outside {GRAD_FROB_BLOCK}; worst " \
+                          f"{np.max(err[live] / nrm[live]) if live.any() else float('nan'):.3e}"
+
+
+def assert_grads_close(got_dH, ref_dH, got_dW, ref_dW):
+    assert frob(got_dH, ref_dH) <= GRAD_FROB
+    assert frob(got_dW, ref_dW) <= GRAD_FROB
+    assert_blocks_close(got_dH, ref_dH, 128, "dH")
+    assert_blocks_close(got_dW, ref_dW, 256, "dW")
+
+
+def oracle_dweight_rows_all_tokens(b, grad_scale, vocab_rows, token_group=128, workers=None):
+    """Rows `vocab_rows` of dW from the oracle, swept over every token that carries loss.
+
+    dW is a sum over tokens.  The sum is taken group by group (the oracle's own `token_group`
+    form of the same sum); here the groups are evaluated by a pool of threads, each calling
+    the oracle on its slice (NumPy releases the interpreter lock inside its loops), and the
+    partial sums are added in token order.  Tokens without loss are left out of the sweep:
+    their logit gradient is exactly zero by definition (pinned in the oracle's own tests)."""
+    import os
+    from concurrent.futures import ThreadPoolExecutor
+    from threadpoolctl import threadpool_limits
+    rows = np.asarray(vocab_rows, dtype=np.int64)
+    W = host(b.weight)
+    idx = torch.nonzero(b.loss_mask != 0).flatten()
+    workers = workers or max(1, (os.cpu_count() or 2) - 1)
+    ones = np.ones(token_group, dtype=np.uint8)
+
+    def part(sl):
+        H, Z = sl
+        return orc.kd_dweight_rows(H, W, Z, ones[: len(H)], b.tau, grad_scale, rows)
+
+    def slices():
+        for i in range(0, idx.numel(), token_group):
+            r = idx[i: i + token_group]
+            yield host(b.hidden[r]), b.teacher[r].float().cpu().numpy()
+
+    out = np.zeros((rows.size, b.d))
+    with threadpool_limits(limits=1), ThreadPoolExecutor(workers) as ex:
+        pending = []
+        for sl in slices():
+            pending.append(ex.submit(part, sl))
+            if len(pending) >= 2 * workers:          # bounded host memory
+                out += pending.pop(0).result()
+        for f in pending:
+            out += f.result()
+    return out
+
+
+def edge_vocab_rows(V, chunk_cols, n, seed):
+    """`n` vocabulary rows: the ends of the 256-wide tiles and of the backward's vocabulary
+    chunks (each boundary and its neighbours), the last rows, and random ones."""
+    rng = np.random.default_rng(seed)
+    fixed = {0, 1, 127, 128, 255, 256, 511, 512, V - 129, V - 128, V - 1}
+    for c in range(chunk_cols, V, chunk_cols):
+        fixed |= {c - 1, c, c + 1}
+    fixed = sorted(r for r in fixed if 0 <= r < V)
+    if len(fixed) > n // 2:                          # many chunks: keep a spread of their edges
+        keep = np.linspace(0, len(fixed) - 1, n // 2).round().astype(int)
+        fixed = sorted({fixed[i] for i in keep} | {0, V - 1})
+    extra = rng.choice(V, size=n, replace=False)
+    rows = list(fixed)
+    for r in extra:
+        if len(rows) >= n:
+            break
+        if int(r) not in rows:
+            rows.append(int(r))
+    return np.asarray(sorted(rows))
 
 
 def assert_losses_close(got, ref, what):
@@ -59,8 +153,7 @@ def check_full_parity(b, step, check_grads=True):
     assert np.all(host(step.kl)[m == 0] == 0)
     if check_grads:
         dH, dW = orc.kd_backward(H, W, Z, m, b.tau, step.grad_scale)
-        assert frob(host(step.d_hidden), dH) <= GRAD_FROB
-        assert frob(host(step.d_weight), dW) <= GRAD_FROB
+        assert_grads_close(host(step.d_hidden), dH, host(step.d_weight), dW)
         assert np.all(host(step.d_hidden)[m == 0] == 0)
     return kl, ns, nt
 

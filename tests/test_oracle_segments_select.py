@@ -271,3 +271,78 @@ def test_packing_invariants_and_quality():
             opt = _min_rows_brute_force(sorted(np.minimum(lengths[want], cap).tolist(), reverse=True), cap)
             rows = len(ptr) - 1
             assert opt <= rows <= (11 * opt + 6) // 9 + 1            # the known first-fit-decreasing bound
+
+
+# --------------------------------------------------------------------------- #
+# Per-sample perplexity (filter ablation, row "Perplexity (PPL)")
+# --------------------------------------------------------------------------- #
+
+def _ppl_table():
+    rows = []
+    with open(os.path.join(os.path.dirname(GOLDEN), "perplexity_table.txt")) as f:
+        for ln in f:
+            if ln.startswith("#") or not ln.strip():
+                continue
+            left, right = ln.split("|")
+            seg, cnt, s = left.split()
+            rows.append((int(seg), int(cnt), float(s), float(right.split()[0])))
+    return rows
+
+
+def test_perplexity_matches_the_hand_worked_table():
+    rows = _ppl_table()
+    cnt = np.asarray([r[1] for r in rows])
+    sums = np.asarray([r[2] for r in rows])
+    want = np.asarray([r[3] for r in rows])
+    got = orc.perplexity_scores(np.arange(len(rows)), sums, cnt)
+    assert np.array_equal(np.isnan(got), np.isnan(want))
+    ok = ~np.isnan(want)
+    assert np.allclose(got[ok], want[ok], rtol=1e-14, atol=0)
+    # the segment index really selects: a permuted request gives the permuted scores
+    perm = np.asarray([5, 0, 3])
+    assert np.allclose(orc.perplexity_scores(perm, sums, cnt), want[perm], rtol=1e-14)
+    # float32 mode: the same two operations in float32
+    g32 = orc.perplexity_scores(np.arange(len(rows)), sums, cnt, dtype=np.float32)
+    assert g32.dtype == np.float32 and np.allclose(g32[ok], want[ok], rtol=1e-6)
+
+
+def test_perplexity_is_the_inverse_geometric_mean_of_the_label_probabilities():
+    # independent restatement: PPL = (prod_t p(y_t))^(-1/n), with the probabilities taken from a
+    # softmax written out here, through the whole chain losses -> segment sums -> score
+    rng = np.random.default_rng(5)
+    T, d, V = 14, 5, 9
+    H, W = rng.standard_normal((T, d)), rng.standard_normal((V, d))
+    Z = rng.standard_normal((T, V))
+    y = rng.integers(0, V, size=T)
+    m = np.ones(T, dtype=np.uint8)
+    cu = np.asarray([0, 5, 6, 14])
+    y[4] = y[5] = y[13] = -100
+    m[[4, 5, 13]] = 0
+    m[7] = 0                                   # a masked token inside a segment
+    kl, ns, nt = orc.kd_token_losses(H, W, Z, y, m, 1.0)
+    _, s_sum, t_sum, cnt = orc.segment_stats(cu, m, y, kl, ns, nt)
+    ppl_s = orc.perplexity_scores([0, 1, 2], s_sum, cnt)
+    ppl_t = orc.perplexity_scores([0, 1, 2], t_sum, cnt)
+    O_S = H @ W.T
+    pS = np.exp(O_S) / np.exp(O_S).sum(1, keepdims=True)
+    pT = np.exp(Z) / np.exp(Z).sum(1, keepdims=True)
+    for s, (a, b) in enumerate(zip(cu[:-1], cu[1:])):
+        tok = [t for t in range(a, b) if m[t] and y[t] >= 0]
+        if not tok:
+            assert np.isnan(ppl_s[s]) and np.isnan(ppl_t[s])
+            continue
+        gs = np.prod([pS[t, y[t]] for t in tok]) ** (-1.0 / len(tok))
+        gt = np.prod([pT[t, y[t]] for t in tok]) ** (-1.0 / len(tok))
+        assert np.isclose(ppl_s[s], gs, rtol=1e-12) and np.isclose(ppl_t[s], gt, rtol=1e-12)
+
+
+def test_perplexity_of_a_uniform_model_is_the_vocabulary_size():
+    T, d, V = 6, 3, 37
+    H, W = np.zeros((T, d)), np.zeros((V, d))          # uniform student
+    Z = np.full((T, V), 0.25)                          # uniform teacher
+    y = np.arange(T) % V
+    m = np.ones(T, dtype=np.uint8)
+    kl, ns, nt = orc.kd_token_losses(H, W, Z, y, m, 1.0)
+    _, s_sum, t_sum, cnt = orc.segment_stats([0, 2, 6], m, y, kl, ns, nt)
+    assert np.allclose(orc.perplexity_scores([0, 1], s_sum, cnt), V, rtol=1e-12)
+    assert np.allclose(orc.perplexity_scores([0, 1], t_sum, cnt), V, rtol=1e-12)
