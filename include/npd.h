@@ -34,12 +34,20 @@
  *   - The caller owns every buffer.  The library allocates no device memory,
  *     keeps no problem state between calls and only enqueues work on the given stream
  *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
- *     Results are ready when the stream has been synchronised.
+ *     Results are ready when the stream has been synchronised.  The exceptions are spelled out
+ *     where they are declared: npd_kd_forward_noalloc works in a fixed array inside the library
+ *     image, and two per-thread diagnostic counters (npd_last_launch_count,
+ *     npd_last_copy_bytes) remember the last call for benchmarks.
  *   - Return value: NPD_OK (0) or a negative npd_status.  Argument errors are
  *     found on the host before anything is launched.  Errors found on the device
  *     (malformed cu_seqlens, a bounded wait that ran out) are recorded in the
  *     workspace and read with npd_last_status().
- *   - No exceptions, no abort(), no device traps.  Device-side waits are bounded.
+ *   - No exceptions, no abort(), no device traps.  Every device-side wait on an mbarrier is
+ *     bounded (about 2 s of SM clocks).  When one runs out the CTA raises an abort flag that all
+ *     its roles poll; warps that meet at named barriers decide together, through a vote at
+ *     such a barrier, whether to go on, so none is left waiting alone; producers give the copies
+ *     they have issued a last bounded grace period to land; both CTAs of a pair meet at the closing
+ *     cluster barrier, tensor memory is freed and the status word reads NPD_ETIMEOUT.
  *   - Needs a device of compute capability 10.x; otherwise NPD_EARCH.
  */
 #ifndef NPD_H_
@@ -78,11 +86,18 @@ enum {
                                outputs are unchanged: the loss value of a token is
                                (1 - lambda) * nll_student[t] + lambda * kl[t].  Without the flag
                                the gradients are those of Eq. 2 alone (lambda = 1). */
-  NPD_KD_REVERSE_KL = 4     /* forward only (d_hidden, d_weight NULL; dense `teacher`): kl[t] becomes
+  NPD_KD_REVERSE_KL = 4,    /* forward only (d_hidden, d_weight NULL; dense `teacher`): kl[t] becomes
                                m_t * D_KL(p_S || p_G) = sum_c p_S(c) (log p_S(c) - log p_G(c)) with
                                p_G = Softmax(teacher[t]/tau), i.e. the divergence of the current
                                learner from the logits of the policy that generated the data, which
                                the paper's appendix tracks as policy lag.  Needs finite logits. */
+  NPD_KD_SERIALIZE_LAUNCHES = 8 /* launch every kernel fully serialised.  By default the tensor-core
+                               kernels of a call are chained as programmatic dependent launches:
+                               the blocks of the next kernel are scheduled, and set up their
+                               barriers and tensor memory, while the last blocks of the kernel
+                               before it are still running, and wait for its completion before
+                               they read or write anything it touches.  Same results either way;
+                               the flag is for debugging and for timing comparisons. */
 };
 
 /*
@@ -267,6 +282,45 @@ int npd_pack_sequences(int32_t N, const int32_t* lengths, const uint8_t* keep, i
                        int32_t* order, int32_t* row_of, int32_t* cu_seqlens, int32_t* row_ptr,
                        int32_t* n_placed, int32_t* n_rows);
 
+/*
+ * Per-sample perplexity, the classical filtering metric that the paper's filter ablation (table
+ * of filtering metrics and selection scopes, row "Perplexity (PPL)") compares Delta-IFD with:
+ *   ppl_X[i] = exp( nll_X_sum[seg[i]] / count[seg[i]] ),   X in {student, teacher},
+ * the exponential of the token-mean cross-entropy of the answer tokens of segment seg[i] (the
+ * per-sequence loss of Eq. 3), in fp32 with IEEE division.  NaN for a sample without such tokens
+ * (count 0) or a segment index outside [0, S).  The paper applies the metric as a weight
+ * ("Weighted" scope) without saying how; only the score is computed here.  Either output (with
+ * its sum array) may be NULL, not both.
+ */
+int npd_perplexity(int32_t N, const int32_t* seg, const float* nll_s_sum, const float* nll_t_sum,
+                   const int32_t* count, int32_t S, float* ppl_student, float* ppl_teacher,
+                   void* cuda_stream);
+
+/*
+ * Self-test of the time-out path (no counterpart in the paper; the failure-handling code of the
+ * tensor kernels would otherwise never run on a healthy device).  Launches one small CTA that
+ * waits, with the same bounded wait and the same group vote the tensor kernels use, on a barrier
+ * nothing arrives on, for `limit_cycles` SM clock cycles (1 .. 1e8; a millisecond is about 2e6).
+ * out3 (DEVICE, int32[3], cleared by the call): [0] the status word, NPD_ETIMEOUT afterwards;
+ * [1] 1 if every thread's wait gave up; [2] cycles thread 0 spent waiting.  No copy or MMA is in
+ * flight in that kernel and it always terminates.
+ */
+int npd_selftest_wait_timeout(int64_t limit_cycles, int32_t* out3, void* cuda_stream);
+
+/*
+ * HOST, diagnostic (no GPU work; no counterpart in the paper).  The units of work CTA pair
+ * `pair` of `pairs` takes in the launch that holds the two backward contractions of one
+ * vocabulary chunk (dW rows of the chunk, and the chunk's contribution to dH): the same
+ * scheduling code the kernel runs, evaluated on the host so that its index arithmetic can be
+ * checked without a device.  row_blocks = blocks of 128 compact rows, d = hidden size,
+ * chunk_cols = vocabulary columns of the chunk.  units (HOST, int32[max_units][5]) receives
+ * {problem (0 = dW, 1 = dH), first row, first column, first k-step, end k-step} per unit, in the
+ * order the pair works through them; *n_units the number of units (also when it exceeds
+ * max_units).
+ */
+int npd_debug_chunk_schedule(int32_t row_blocks, int32_t d, int32_t chunk_cols, int32_t pairs,
+                             int32_t pair, int32_t max_units, int32_t* units, int32_t* n_units);
+
 /* Synchronises `cuda_stream`, then reads the device-side status word of a
  * workspace that npd_kd_fwd_bwd used into *host_status (HOST): NPD_OK,
  * NPD_ESEQ or NPD_ETIMEOUT.  Returns NPD_ECUDA if the stream itself failed. */
@@ -275,12 +329,13 @@ int npd_last_status(const void* workspace, void* cuda_stream, int32_t* host_stat
 /* HOST.  Static description of a status code. */
 const char* npd_strerror(int status);
 
-/* HOST.  Number of kernel launches the last npd_kd_fwd_bwd call on this thread
- * enqueued (for launch accounting in benchmarks). */
+/* HOST, diagnostic.  Number of kernel launches the last npd_kd_fwd_bwd call on this thread
+ * enqueued (for launch accounting in benchmarks).  One of the two pieces of per-thread state
+ * the library keeps; it influences nothing. */
 int npd_last_launch_count(void);
 
-/* HOST.  Bytes the last npd_kd_fwd_bwd_host call on this thread copied host-to-device and
- * device-to-host. */
+/* HOST, diagnostic.  Bytes the last npd_kd_fwd_bwd_host call on this thread copied
+ * host-to-device and device-to-host (per-thread state like the launch count). */
 int npd_last_copy_bytes(int64_t* h2d_bytes, int64_t* d2h_bytes);
 
 /*

@@ -23,6 +23,7 @@ NPD_DTYPE_BF16, NPD_DTYPE_F32 = 0, 1
 NPD_KD_ACCUMULATE_DW = 1
 NPD_KD_COMPOSITE_LOSS = 2
 NPD_KD_REVERSE_KL = 4
+NPD_KD_SERIALIZE_LAUNCHES = 8
 NPD_SELECT_TEACHER_IFD_LE_1 = 1
 NPD_SELECT_SCORE_IFD_TEACHER, NPD_SELECT_SCORE_IFD_STUDENT = 2, 4
 NPD_SELECT_LO_EXCLUSIVE, NPD_SELECT_HI_EXCLUSIVE = 8, 16
@@ -31,7 +32,8 @@ NPD_GEMM_STORE_F32, NPD_GEMM_ADD_F32, NPD_GEMM_STORE_BF16, NPD_GEMM_ATOMIC_F32 =
 EXPORTS = ("npd_workspace_bytes", "npd_phase_count", "npd_kd_fwd_bwd", "npd_kd_fwd_bwd_host", "npd_segment_stats",
            "npd_select", "npd_last_status", "npd_strerror", "npd_last_launch_count", "npd_gemm_bf16",
            "npd_kd_forward_noalloc", "npd_pack_sequences", "npd_last_copy_bytes",
-           "npd_kd_fwd_bwd_host_streams")
+           "npd_kd_fwd_bwd_host_streams", "npd_perplexity", "npd_selftest_wait_timeout",
+           "npd_debug_chunk_schedule")
 NPD_STATIC_SCRATCH_BYTES = 48 * 1024 * 1024
 
 
@@ -95,6 +97,9 @@ def lib() -> C.CDLL:
         l.npd_last_copy_bytes.argtypes = [C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         l.npd_kd_forward_noalloc.argtypes = [C.POINTER(npd_kd_args), C.c_void_p, C.POINTER(C.c_int32)]
         l.npd_pack_sequences.argtypes = [C.c_int32, C.c_void_p, C.c_void_p, C.c_int32] + [C.c_void_p] * 6
+        l.npd_perplexity.argtypes = [C.c_int32] + [C.c_void_p] * 4 + [C.c_int32] + [C.c_void_p] * 3
+        l.npd_selftest_wait_timeout.argtypes = [C.c_int64, C.c_void_p, C.c_void_p]
+        l.npd_debug_chunk_schedule.argtypes = [C.c_int32] * 6 + [C.c_void_p, C.POINTER(C.c_int32)]
         l.npd_gemm_bf16.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_int64, C.c_int32,
                                     C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64,
                                     C.c_int32, C.c_int32, C.c_void_p]
@@ -245,6 +250,41 @@ def npd_select(cond_seg, uncond_seg, nll_s_sum, nll_t_sum, count, lo: float, hi:
                             _ptr(count), S, float(lo), float(hi), int(flags), _ptr(ifd_t), _ptr(ifd_s),
                             _ptr(delta), _ptr(keep), _ptr(n_keep), _stream(stream)), "npd_select")
     return ifd_t, ifd_s, delta, keep, n_keep
+
+
+def npd_perplexity(seg, nll_s_sum, nll_t_sum, count, stream=None):
+    """Per-sample perplexities exp(nll_sum / count) of the segments `seg`.  Returns
+    (ppl_student, ppl_teacher); an output is None when its sums are None."""
+    N, S, dev = seg.numel(), count.numel(), seg.device
+    ps = torch.empty(N, dtype=torch.float32, device=dev) if nll_s_sum is not None else None
+    pt = torch.empty(N, dtype=torch.float32, device=dev) if nll_t_sum is not None else None
+    _check(lib().npd_perplexity(N, _ptr(seg), _ptr(nll_s_sum), _ptr(nll_t_sum), _ptr(count), S, _ptr(ps),
+                                _ptr(pt), _stream(stream)), "npd_perplexity")
+    return ps, pt
+
+
+def npd_selftest_wait_timeout(limit_cycles: int, device="cuda", stream=None):
+    """Runs the time-out path of the bounded device waits on purpose (see include/npd.h).
+    Returns the int32[3] device tensor {status, every wait gave up, cycles waited}."""
+    out = torch.empty(3, dtype=torch.int32, device=device)
+    _check(lib().npd_selftest_wait_timeout(int(limit_cycles), _ptr(out), _stream(stream)),
+           "npd_selftest_wait_timeout")
+    return out
+
+
+def npd_debug_chunk_schedule(row_blocks: int, d: int, chunk_cols: int, pairs: int, pair: int):
+    """Host only: the (problem, row, column, k-step begin, k-step end) units of one CTA pair in the
+    launch of a chunk's two backward contractions, as an int32 array [n, 5]."""
+    import numpy as np
+    n = C.c_int32(0)
+    cap = 64
+    while True:
+        units = np.empty((cap, 5), np.int32)
+        _check(lib().npd_debug_chunk_schedule(row_blocks, d, chunk_cols, pairs, pair, cap, units.ctypes.data,
+                                              C.byref(n)), "npd_debug_chunk_schedule")
+        if n.value <= cap:
+            return units[: n.value].copy()
+        cap = n.value
 
 
 def npd_pack_sequences(lengths, keep, capacity: int):

@@ -8,12 +8,17 @@
 // (memory [K][rows contiguous]); the second form lets the logit-gradient block
 // and the hidden states be read as they lie in memory, with no transposes.
 //
-// One launch runs one or two such problems.  With two, the CTA pairs first take the
-// units (whole tiles) of problem 0 round robin; problem 1 is then laid out as one long line
-// of (tile, k-step) positions and every pair gets the stretch of that line that brings it to
-// the same total number of k-steps as all the others (a stretch may start and end in the
-// middle of a tile: the pieces are added with fp32 atomics).  This is how the dW and dH
-// products of one vocabulary chunk share a launch and end together.
+// One launch runs one or two such problems.  With two (the dW and dH products of one vocabulary
+// chunk, which share N = d) the CTA pairs work in groups of as many pairs as a row tile has
+// 512-wide column tiles: the members of a group take the column tiles of the SAME row tile at the
+// same time, so the A operand they share (a panel of the logit-gradient block) is fetched from
+// HBM once and served to the others from L2.  A group first takes whole row tiles of problem 0
+// (last row tiles first: they are the part of the gradient block written last, still in L2);
+// problem 1 is then laid out as one long line of (row tile, k-step) positions and every group gets
+// the stretch of that line that brings it to the same total number of k-steps as all the others
+// (a stretch may start and end in the middle of a tile: the pieces are added with fp32 atomics).
+// Pairs that do not fill a group take whole tiles of problem 0 only.  This is how the two
+// products share a launch and end together.
 //
 // Two CTAs on neighbouring SMs (a cluster of 2) work as a pair on a 256 x 512 output tile
 // with tcgen05 .cta_group::2 (two M=256, N=256 accumulators that share the A operand): per
@@ -81,7 +86,7 @@ struct GemmUnit {
   int ns;                // accumulators in use: 2, or 1 when the tile's second 256 columns lie beyond N
 };
 // Tile `tile` (n fastest) of a problem, k-tiles [kt0, kt1).
-__device__ __forceinline__ GemmUnit gemm_tile_unit(const GemmProblem& g, int tile, int kt0, int kt1) {
+__host__ __device__ __forceinline__ GemmUnit gemm_tile_unit(const GemmProblem& g, int tile, int kt0, int kt1) {
   using namespace gemm_cfg;
   const int tiles_n = (g.N + BN - 1) / BN;
   GemmUnit u;
@@ -98,22 +103,71 @@ struct GemmWalk {
   GemmProblem pr[2];
   int c, C;            // this pair and the number of pairs
   int tiles[2], ksteps[2];
-  int i;               // units taken so far in the round-robin phases
+  int i;               // units taken so far in the whole-tile phases
   long long pos, end;  // problem 1 with stream_k: this pair's stretch of the (tile, k-step) line
+  // grouped mode (two problems that share N; see the head of this file)
+  int grouped;
+  int tn;              // column tiles per row tile = pairs per group
+  int G;               // number of groups; pairs G*tn .. C-1 stand outside the groups
+  int g, j;            // this pair's group and its column tile (g == G: outside the groups)
+  int mt0, m_lone;     // row tiles of problem 0; the first m_lone of them go to the lone pairs
+  int mine0;           // units of problem 0 this pair takes
+  int lone_first;      // lone pair: its first tile (n fastest) of problem 0
 
-  __device__ __forceinline__ void init(const GemmParams& p, int c_, int C_) {
+  // nb = number of 128-row blocks behind the device-side extents (dyn_m / dyn_k)
+  __host__ __device__ __forceinline__ void init(const GemmParams& p, int nb, int c_, int C_) {
     using namespace gemm_cfg;
     c = c_;
     C = C_;
     i = 0;
     pos = end = 0;
+    grouped = 0;
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
       pr[q] = p.pr[q];
-      if (pr[q].dyn_m) pr[q].M = 128 * __ldg(p.nblocks);
-      if (pr[q].dyn_k) pr[q].K = 128 * __ldg(p.nblocks);
+      if (pr[q].dyn_m) pr[q].M = 128 * nb;
+      if (pr[q].dyn_k) pr[q].K = 128 * nb;
       tiles[q] = q < p.nprob ? ((pr[q].M + PM - 1) / PM) * ((pr[q].N + BN - 1) / BN) : 0;
       ksteps[q] = (pr[q].K + BK - 1) / BK;
+    }
+    tn = (pr[0].N + BN - 1) / BN;
+    G = tn > 0 ? C / tn : 0;
+    if (p.nprob == 2 && pr[1].stream_k && pr[0].k_splits == 1 && pr[0].N == pr[1].N && G > 0 &&
+        tiles[0] > 0 && tiles[1] > 0 && ksteps[0] > 0 && ksteps[1] > 0) {
+      grouped = 1;
+      mt0 = tiles[0] / tn;
+      const int mt1 = tiles[1] / tn;
+      const int lone = C - G * tn;
+      const double k0 = ksteps[0];
+      const double line = static_cast<double>(mt1) * ksteps[1];
+      // lone pairs: whole tiles of problem 0, no more than an even share of the launch's k-steps
+      m_lone = 0;
+      if (lone > 0) {
+        const double share = (static_cast<double>(tiles[0]) * k0 + line * tn) / C;
+        const int per = static_cast<int>(share / k0);
+        m_lone = mt0 < lone * per / tn ? mt0 : lone * per / tn;
+      }
+      const int R = mt0 - m_lone;  // row tiles of problem 0 the groups take, round robin
+      g = c / tn;
+      j = c - g * tn;
+      if (g >= G) {
+        g = G;
+        const int l = c - G * tn, xl = m_lone * tn, per = xl / lone, extra = xl % lone;
+        lone_first = l * per + (l < extra ? l : extra);
+        mine0 = per + (l < extra ? 1 : 0);
+      } else {
+        const int q0 = R / G, rem0 = R % G;
+        mine0 = q0 + (g < rem0 ? 1 : 0);
+        // groups 0..rem0-1 hold one more row tile of problem 0 and get the shorter stretch sa
+        const double target = (R * k0 + line) / G;
+        double sa = target - (q0 + 1) * k0;
+        sa = sa > 0.0 ? sa : 0.0;
+        const double sb = rem0 < G ? (line - rem0 * sa) / (G - rem0) : 0.0;
+        auto prefix = [&](int k) { return k <= rem0 ? k * sa : rem0 * sa + (k - rem0) * sb; };
+        pos = static_cast<long long>(prefix(g) + 0.5);
+        end = g + 1 == G ? static_cast<long long>(line) : static_cast<long long>(prefix(g + 1) + 0.5);
+      }
+      return;
     }
     if (tiles[1] > 0 && pr[1].stream_k && ksteps[1] > 0) {
       // k-steps of problem 0 this pair and its neighbours carry (units go round robin)
@@ -131,10 +185,29 @@ struct GemmWalk {
     }
   }
 
-  __device__ __forceinline__ bool next(int& prob, GemmUnit& u) {
+  __host__ __device__ __forceinline__ bool next(int& prob, GemmUnit& u) {
+    if (grouped) {
+      if (i < mine0) {
+        prob = 0;
+        // lone pair: consecutive tiles; group member: its column tile of the group's i-th row tile,
+        // the last row tiles first
+        const int tile = g == G ? lone_first + i : (mt0 - 1 - (g + i * G)) * tn + j;
+        u = gemm_tile_unit(pr[0], tile, 0, ksteps[0]);
+        ++i;
+        return true;
+      }
+      prob = 1;
+      if (pos >= end) return false;
+      const int m = static_cast<int>(pos / ksteps[1]), k0 = static_cast<int>(pos % ksteps[1]);
+      const long long left = end - pos;
+      const int len = left < ksteps[1] - k0 ? static_cast<int>(left) : ksteps[1] - k0;
+      u = gemm_tile_unit(pr[1], m * tn + j, k0, k0 + len);
+      pos += len;
+      return true;
+    }
     const int units0 = tiles[0] * pr[0].k_splits;
-    const int mine0 = units0 / C + (c < units0 % C ? 1 : 0);
-    if (i < mine0) {
+    const int mine = units0 / C + (c < units0 % C ? 1 : 0);
+    if (i < mine) {
       const int v = c + i * C, ks = v / tiles[0];
       prob = 0;
       u = gemm_tile_unit(pr[0], v % tiles[0],
@@ -153,7 +226,7 @@ struct GemmWalk {
       pos += len;
       return true;
     }
-    const int v = c + (i - mine0) * C;
+    const int v = c + (i - mine) * C;
     if (v >= tiles[1] * pr[1].k_splits) return false;
     const int ks = v / tiles[1];
     u = gemm_tile_unit(pr[1], v % tiles[1],
@@ -216,8 +289,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
   const uint32_t tempty_leader = mapa_shared(tempty, 0);
 
   // every role resolves the same problems and walks the same sequence of units
+  // (the extents may come from the kernel before this one in the stream)
+  grid_dependency_wait();
+  grid_launch_dependents();
   GemmWalk walk;
-  walk.init(p, cluster_id, num_clusters);
+  const bool dyn = p.pr[0].dyn_m || p.pr[0].dyn_k || p.pr[1].dyn_m || p.pr[1].dyn_k;
+  walk.init(p, dyn ? __ldg(p.nblocks) : 0, cluster_id, num_clusters);
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
@@ -263,9 +340,22 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
       // Drain: a stage is released only after its loads landed and the MMAs that read it
       // finished, so waiting for the release of the last stages covers both.
       const uint32_t last = it < STAGES ? it : STAGES;
-      for (uint32_t j = 0; j < last; ++j) {
+      for (uint32_t j = 0; j < last && ok; ++j) {
         const uint32_t i2 = it - 1 - j;
-        mbar_wait(empty0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1, abort_flag);
+        ok = mbar_wait(empty0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1, abort_flag);
+      }
+      if (!ok) {
+        // Aborted: nobody may be left to release the stages, but the loads already issued still
+        // land in this CTA's shared memory.  The leader's "full" barriers count both CTAs' bytes;
+        // the peer cannot wait on them and lets the grace period pass instead.
+        if (rank == 0) {
+          for (uint32_t j = 0; j < last; ++j) {
+            const uint32_t i2 = it - 1 - j;
+            mbar_wait_drain(full0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1);
+          }
+        } else {
+          grace_sleep();
+        }
       }
     }
   } else if (warp == 1) {
@@ -331,7 +421,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
       // sub-tiles of this group that lie inside N (uniform over the group)
       int nsteps = (g.N - (u.n0 + c0) + step - 1) / step;
       nsteps = nsteps < 0 ? 0 : (nsteps > gcols / step ? gcols / step : nsteps);
-      ok = __all_sync(0xffffffffu, mbar_wait(tfull, tile & 1, abort_flag));
+      // the four warps of a group stay or leave together (they meet at barriers below)
+      ok = named_barrier_vote(bar_id, 128, __all_sync(0xffffffffu, mbar_wait(tfull, tile & 1, abort_flag)));
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + c0;

@@ -183,6 +183,12 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   const uint32_t full_leader = mapa_shared(full0, 0);
   const uint32_t tempty_leader = mapa_shared(tempty0, 0);
 
+  // Everything above touched only this CTA's own resources.  What follows reads what earlier
+  // kernels in the stream wrote (the plan, the compact rows, the log-sum-exps) and overwrites
+  // what they read (the gradient scratch), so it waits for them to be complete.
+  grid_dependency_wait();
+  grid_launch_dependents();
+
   const int nact = p.plan[0], pairs = p.plan[1];
   const int nsplit = kMode == kForward ? p.plan[2] : p.vt_count;
   const int units = pairs * nsplit;
@@ -224,9 +230,22 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       // Drain: a stage is released only after its loads landed and the MMAs that read it
       // finished, so waiting for the release of the last stages covers both.
       const uint32_t last = it < STAGES ? it : STAGES;
-      for (uint32_t j = 0; j < last; ++j) {
+      for (uint32_t j = 0; j < last && ok; ++j) {
         const uint32_t i2 = it - 1 - j;
-        mbar_wait(empty0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1, abort_flag);
+        ok = mbar_wait(empty0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1, abort_flag);
+      }
+      if (!ok) {
+        // Aborted: nobody may be left to release the stages, but the loads already issued still
+        // land in this CTA's shared memory.  The leader's "full" barriers count both CTAs' bytes;
+        // the peer cannot wait on them and lets the grace period pass instead.
+        if (rank == 0) {
+          for (uint32_t j = 0; j < last; ++j) {
+            const uint32_t i2 = it - 1 - j;
+            mbar_wait_drain(full0 + 8 * (i2 % STAGES), (i2 / STAGES) & 1);
+          }
+        } else {
+          grace_sleep();
+        }
       }
     }
   } else if (warp == 1) {
@@ -292,11 +311,15 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           }
         }
       }
-      const uint32_t last = zit < ZQ ? zit : ZQ;
+      // Every gather issued must have landed before this CTA's shared memory is given up.  After
+      // an abort the sub-tile pair that was being issued may be half out, so it is included; a
+      // stage that was never armed just lets its (short) limit pass.
+      const uint32_t upto = ok ? zit : zit + 1;
+      const uint32_t last = upto < ZQ ? upto : ZQ;
       for (uint32_t j = 0; j < last; ++j) {
-        const uint32_t i2 = zit - 1 - j;
+        const uint32_t i2 = upto - 1 - j;
         for (int half = 0; half < 2; ++half)
-          mbar_wait(zfull0 + 8 * (half * ZQ + (i2 % ZQ)), (i2 / ZQ) & 1, abort_flag);
+          mbar_wait_drain(zfull0 + 8 * (half * ZQ + (i2 % ZQ)), (i2 / ZQ) & 1);
       }
     }
   } else if (warp >= 4) {
@@ -342,8 +365,12 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       }
       for (int vt = vt0; vt < vt1 && ok; ++vt, ++tile) {
         const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
-        ok = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * buf, tph, abort_flag));
-        if (!ok) break;
+        // okw: this warp's waits so far succeeded.  In the forward pass a warp that gives up just
+        // leaves.  In the gradient pass the four warps of a column half meet at named barriers, so
+        // a warp whose wait ran out keeps joining them (doing nothing else) until the vote at the
+        // end of the sub-tile tells the whole half to leave together.
+        bool okw = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * buf, tph, abort_flag));
+        if (kMode == kForward && !okw) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t taddr =
             tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN + half * (BN / 2);
@@ -351,13 +378,14 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           const uint32_t q = zit % ZQ, zph = (zit / ZQ) & 1;
           const uint32_t bi = 8 * (half * ZQ + q);
           if (!kSparse) {
-            ok = __all_sync(0xffffffffu, mbar_wait(zfull0 + bi, zph, abort_flag));
-            if (!ok) break;
+            okw = okw && __all_sync(0xffffffffu, mbar_wait(zfull0 + bi, zph, abort_flag));
+            if (kMode == kForward && !okw) { ok = false; break; }
           }
+          if (kMode == kGradient && kTeacherF32 && !okw) named_barrier_sync(1 + half, 128);  // see below
           uint8_t* zrow = smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES + row_local * 128;
           const int sub_col0 = vt * BN + half * (BN / 2) + j * ZC;
 #pragma unroll 1
-          for (int c = 0; c < ZC / 32; ++c) {
+          for (int c = 0; okw && c < ZC / 32; ++c) {
             const int col0 = sub_col0 + c * 32;
             uint32_t acc[32];
             tmem_ld32(taddr + j * ZC + c * 32, acc);
@@ -508,7 +536,8 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           } else {
             // hand the finished 128 x 64 gradient sub-tile to TMA, then recycle the stage
             fence_proxy_async_smem();
-            named_barrier_sync(1 + half, 128);
+            ok = named_barrier_vote(1 + half, 128, okw);
+            if (!ok) break;
             if (lg == 0 && lane == 0) {
               if (r >= 0) {
                 tma_store_2d(&tmap_g, smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES),

@@ -187,11 +187,40 @@ struct PhaseRecorder {
   }
 };
 
+// Raises a kernel's dynamic shared-memory limit; done once per kernel and device.
 template <typename K>
 int set_smem(K kernel, int bytes) {
-  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess
-             ? NPD_OK
-             : NPD_ECUDA;
+  static std::mutex mu;
+  static std::vector<std::pair<const void*, int>> done;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return NPD_ECUDA;
+  const void* key = reinterpret_cast<const void*>(kernel);
+  std::lock_guard<std::mutex> lock(mu);
+  for (const auto& e : done)
+    if (e.first == key && e.second == dev) return NPD_OK;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess)
+    return NPD_ECUDA;
+  done.emplace_back(key, dev);
+  return NPD_OK;
+}
+
+// Launch with (pdl) or without the programmatic-dependent-launch attribute: with it, the blocks
+// of this kernel may be scheduled and run their prologue while the kernel before it in the stream
+// is still draining; they wait for that kernel's completion inside (griddepcontrol.wait).
+template <typename... P, typename... A>
+cudaError_t launch_ex(void (*kernel)(P...), int grid, int threads, int smem, cudaStream_t st, bool pdl,
+                      A&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3(static_cast<unsigned>(threads));
+  cfg.dynamicSmemBytes = static_cast<size_t>(smem);
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
 }
 
 struct GemmOperands {
@@ -203,10 +232,36 @@ struct GemmOperands {
   long long ldo;
 };
 
+// The two backward contractions of one vocabulary chunk of `cols` columns.  Everything lives on
+// the compact rows (their number is only known on the device): the logit-gradient block, the
+// gathered hidden states and the fp32 dH accumulator.
+void chunk_problems(int d, int cols, bool dw_f32, bool dw_accumulate, GemmProblem* pr) {
+  // dW[col0 .. col0+cols) = G_chunk^T Hc      (M = vocabulary rows, N = d, K = compact rows)
+  pr[0] = GemmProblem{};
+  pr[0].M = cols;
+  pr[0].N = d;
+  pr[0].dyn_k = 1;
+  pr[0].a_mn = 1;
+  pr[0].b_mn = 1;
+  pr[0].k_splits = 1;
+  pr[0].out_f32 = dw_f32;
+  pr[0].out_reduce = dw_accumulate ? 1 : 0;
+  // dH += G_chunk W[col0 .. col0+cols)        (M = compact rows, N = d, K = the chunk's columns)
+  pr[1] = GemmProblem{};
+  pr[1].dyn_m = 1;
+  pr[1].N = d;
+  pr[1].K = cols;
+  pr[1].b_mn = 1;
+  pr[1].k_splits = 1;
+  pr[1].stream_k = 1;
+  pr[1].out_f32 = 1;
+  pr[1].out_reduce = 1;
+}
+
 // One launch for one or two problems (see gemm_sm100.cuh for how the units are dealt).
 // An extent only known on the device (dyn_m / dyn_k) is 128 * max_blocks as far as the maps go.
 int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const int* nblocks,
-                int max_blocks, int* status, int sms, cudaStream_t st) {
+                int max_blocks, int* status, int sms, cudaStream_t st, bool pdl = false) {
   using namespace gemm_cfg;
   CUtensorMap maps[6];
   GemmParams gp{};
@@ -234,15 +289,15 @@ int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const
   gp.status = status;
   const int pairs = static_cast<int>(std::max<long long>(1, std::min<long long>(units, std::max(sms / 2, 1))));
   if (set_smem(gemm_bf16_kernel, SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
-  gemm_bf16_kernel<<<2 * pairs, THREADS, SMEM_BYTES, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4],
-                                                          maps[5], gp);
+  const cudaError_t e = launch_ex(gemm_bf16_kernel, 2 * pairs, THREADS, SMEM_BYTES, st, pdl, maps[0], maps[1],
+                                  maps[2], maps[3], maps[4], maps[5], gp);
   ++g_launches;
-  return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
+  return e == cudaSuccess ? NPD_OK : NPD_ECUDA;
 }
 
 template <int kMode>
 int launch_kd_tile(bool tau_one, bool composite, bool sparse, bool tf32, const CUtensorMap& mh, const CUtensorMap& mw, const CUtensorMap& mt,
-                   const CUtensorMap& mg, const KdTileParams& kp, int sms, cudaStream_t st) {
+                   const CUtensorMap& mg, const KdTileParams& kp, int sms, cudaStream_t st, bool pdl) {
   using namespace kd_cfg;
   composite = composite && kMode == kGradient;  // the forward does not depend on the objective's mix
   auto k = kd_tile_kernel<kMode, true, false, false, false>;
@@ -259,9 +314,9 @@ int launch_kd_tile(bool tau_one, bool composite, bool sparse, bool tf32, const C
   if (set_smem(k, Layout<kMode>::SMEM_BYTES) != NPD_OK) return NPD_ECUDA;
   // the number of units is only known on the device: always one CTA pair per two SMs
   const int grid = 2 * std::max(sms / 2, 1);
-  k<<<grid, THREADS, Layout<kMode>::SMEM_BYTES, st>>>(mh, mw, mt, mg, kp);
+  const cudaError_t e = launch_ex(k, grid, THREADS, Layout<kMode>::SMEM_BYTES, st, pdl, mh, mw, mt, mg, kp);
   ++g_launches;
-  return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
+  return e == cudaSuccess ? NPD_OK : NPD_ECUDA;
 }
 
 }  // namespace
@@ -335,6 +390,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   if (cudaMemsetAsync(status, 0, 64, st) != cudaSuccess) return NPD_ECUDA;
   PhaseRecorder rec{a->phase_events, a->n_phase_events, 0, st};
 
+  const bool pdl = (a->flags & NPD_KD_SERIALIZE_LAUNCHES) == 0;
   const bool tau_one = a->temperature == 1.0f;
   const float scale2 = 1.4426950408889634f / a->temperature;
 
@@ -386,7 +442,7 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
   kp.partials = partials;
   kp.reverse = (a->flags & NPD_KD_REVERSE_KL) ? 1 : 0;
   kp.status = status;
-  if ((rc = launch_kd_tile<kForward>(tau_one, false, sparse, tf32, mh, mw, mt, mt, kp, di.sms, st)) != NPD_OK) return rc;
+  if ((rc = launch_kd_tile<kForward>(tau_one, false, sparse, tf32, mh, mw, mt, mt, kp, di.sms, st, pdl)) != NPD_OK) return rc;
   rec.mark();
 
   if (sparse) {
@@ -492,42 +548,20 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     gp.tk_cp = tk_cp;
     gp.topk = a->topk;
     gp.g_col0 = col0;
-    if ((rc = launch_kd_tile<kGradient>(tau_one, composite, sparse, tf32, mh, mw, mt, mg, gp, di.sms, st)) != NPD_OK) return rc;
+    if ((rc = launch_kd_tile<kGradient>(tau_one, composite, sparse, tf32, mh, mw, mt, mg, gp, di.sms, st, pdl)) != NPD_OK) return rc;
     rec.mark();
 
     GemmProblem pr[2] = {};
     GemmOperands ops[2] = {};
-    // Everything here lives on the compact rows: the logit-gradient block, the gathered hidden
-    // states and the fp32 dH accumulator.
-    // dW[col0 .. col0+cols) = G_chunk^T Hc      (M = vocabulary rows, N = d, K = compact rows)
-    pr[0].M = cols;
-    pr[0].N = a->d;
-    pr[0].K = 0;
-    pr[0].dyn_k = 1;
-    pr[0].a_mn = 1;
-    pr[0].b_mn = 1;
-    pr[0].k_splits = 1;
-    pr[0].out_f32 = a->d_weight_dtype == NPD_DTYPE_F32;
-    pr[0].out_reduce = (a->flags & NPD_KD_ACCUMULATE_DW) ? 1 : 0;
+    chunk_problems(a->d, cols, a->d_weight_dtype == NPD_DTYPE_F32, (a->flags & NPD_KD_ACCUMULATE_DW) != 0, pr);
     void* dw_rows = pr[0].out_f32
                         ? static_cast<void*>(static_cast<float*>(a->d_weight) + static_cast<size_t>(col0) * a->ldw)
                         : static_cast<void*>(static_cast<__nv_bfloat16*>(a->d_weight) +
                                              static_cast<size_t>(col0) * a->ldw);
     ops[0] = {gbuf, ldg, hc, a->d, dw_rows, a->ldw};
-    // dH += G_chunk W[col0 .. col0+cols)        (M = compact rows, N = d, K = the chunk's columns)
-    pr[1].M = 0;
-    pr[1].dyn_m = 1;
-    pr[1].N = a->d;
-    pr[1].K = cols;
-    pr[1].a_mn = 0;
-    pr[1].b_mn = 1;
-    pr[1].k_splits = 1;
-    pr[1].stream_k = 1;
-    pr[1].out_f32 = 1;
-    pr[1].out_reduce = 1;
     const __nv_bfloat16* w_rows = static_cast<const __nv_bfloat16*>(a->weight) + static_cast<size_t>(col0) * a->ldw;
     ops[1] = {gbuf, ldg, w_rows, a->ldw, dh_acc, a->d};
-    if ((rc = launch_gemm(2, pr, ops, plan, pl.row_blocks, status, di.sms, st)) != NPD_OK) return rc;
+    if ((rc = launch_gemm(2, pr, ops, plan, pl.row_blocks, status, di.sms, st, pdl)) != NPD_OK) return rc;
     rec.mark();
   }
   {
@@ -732,6 +766,54 @@ int npd_pack_sequences(int32_t N, const int32_t* lengths, const uint8_t* keep, i
   row_ptr[members.size()] = j;
   *n_placed = j;
   *n_rows = static_cast<int32_t>(members.size());
+  return NPD_OK;
+}
+
+int npd_perplexity(int32_t N, const int32_t* seg, const float* nll_s_sum, const float* nll_t_sum,
+                   const int32_t* count, int32_t S, float* ppl_student, float* ppl_teacher,
+                   void* cuda_stream) {
+  if (N < 1 || S < 1 || seg == nullptr || count == nullptr) return NPD_EINVAL;
+  if ((ppl_student != nullptr && nll_s_sum == nullptr) || (ppl_teacher != nullptr && nll_t_sum == nullptr) ||
+      (ppl_student == nullptr && ppl_teacher == nullptr))
+    return NPD_EINVAL;
+  perplexity_kernel<<<(N + 255) / 256, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      N, S, seg, nll_s_sum, nll_t_sum, count, ppl_student, ppl_teacher);
+  return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
+}
+
+int npd_selftest_wait_timeout(int64_t limit_cycles, int32_t* out3, void* cuda_stream) {
+  // the limit is kept short on purpose: this entry point exists to run the time-out path, not to wait
+  if (out3 == nullptr || limit_cycles < 1 || limit_cycles > 100000000) return NPD_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(out3, 0, 3 * sizeof(int32_t), st) != cudaSuccess) return NPD_ECUDA;
+  wait_timeout_selftest_kernel<<<1, 128, 0, st>>>(static_cast<long long>(limit_cycles), out3);
+  return cudaGetLastError() == cudaSuccess ? NPD_OK : NPD_ECUDA;
+}
+
+int npd_debug_chunk_schedule(int32_t row_blocks, int32_t d, int32_t chunk_cols, int32_t pairs, int32_t pair,
+                             int32_t max_units, int32_t* units, int32_t* n_units) {
+  if (row_blocks < 0 || d < 1 || chunk_cols < 1 || pairs < 1 || pair < 0 || pair >= pairs || max_units < 0 ||
+      n_units == nullptr || (max_units > 0 && units == nullptr))
+    return NPD_EINVAL;
+  GemmParams gp{};
+  chunk_problems(d, chunk_cols, false, false, gp.pr);
+  gp.nprob = 2;
+  GemmWalk walk;
+  walk.init(gp, row_blocks, pair, pairs);
+  int n = 0, prob = 0;
+  GemmUnit u;
+  while (walk.next(prob, u)) {
+    if (n < max_units) {
+      int32_t* o = units + 5 * n;
+      o[0] = prob;
+      o[1] = u.m0;
+      o[2] = u.n0;
+      o[3] = u.kt0;
+      o[4] = u.kt1;
+    }
+    ++n;
+  }
+  *n_units = n;
   return NPD_OK;
 }
 

@@ -62,21 +62,43 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  Returns false when the limit ran out or another thread of the
-// CTA already gave up (*abort_flag != 0); the caller then leaves its role loop.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// Bounded wait.  Returns false when the limit (in SM clock cycles) ran out or another thread of
+// the CTA already gave up (*abort_flag != 0); the caller then leaves its role loop.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 0xFF) == 0) {
+    // a failing try_wait already suspends the thread for a few microseconds, so a look at the
+    // flag and the clock every 16 of them keeps the limit accurate to a fraction of a millisecond
+    if ((it & 0xF) == 0) {
       if (*abort_flag != 0) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit_cycles) {
         *abort_flag = 1;
         return false;
       }
     }
   }
+}
+
+// Grace period of a producer that leaves after an abort: copies it has issued complete on their
+// own, so their barrier is waited for once more, for at most this many cycles (about 1 ms),
+// whatever the abort flag says.
+constexpr long long kDrainLimitCycles = 2000000LL;
+__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 0xF) == 0 && clock64() - t0 > kDrainLimitCycles) return false;
+  }
+}
+// The same grace period where the copies signal a barrier this thread cannot wait on (one that
+// lives in the peer CTA): just let the time pass.
+__device__ __forceinline__ void grace_sleep() {
+  const long long t0 = clock64();
+  while (clock64() - t0 < kDrainLimitCycles) __nanosleep(256);
 }
 
 // ----------------------------------------------------------------------------
@@ -298,6 +320,31 @@ __device__ __forceinline__ float lg2f(float x) {
 }
 __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// Barrier over `nthreads` threads that also returns the AND of everybody's `ok`: the way a group
+// of warps decides together whether to go on, so that none of them is left alone at a later
+// barrier after a wait ran out for some of them only.
+__device__ __forceinline__ bool named_barrier_vote(int id, int nthreads, bool ok) {
+  uint32_t all;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %3, 0;\n\t"
+      "barrier.cta.red.and.pred p, %1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(all)
+      : "r"(id), "r"(nthreads), "r"(static_cast<uint32_t>(ok))
+      : "memory");
+  return all != 0;
+}
+// Programmatic dependent launch.  launch_dependents: the next kernel in the stream may start
+// being scheduled (its blocks still wait in grid_dependency_wait for this grid to finish and
+// flush).  grid_dependency_wait: returns once the preceding grid has completed and its writes
+// are visible; a no-op when the kernel was not launched as a dependent.
+__device__ __forceinline__ void grid_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);

@@ -449,6 +449,56 @@ __global__ void __launch_bounds__(256) select_kernel(
   if ((threadIdx.x & 31) == 0 && kept != 0) atomicAdd(n_keep, kept);
 }
 
+// One thread per sample: perplexity of the sample's answer tokens under the student and under the
+// teacher, exp(token-mean cross-entropy) (the classical filtering metric the filter ablation
+// compares Delta-IFD with); NaN for a sample without such tokens or a segment index out of range.
+__global__ void __launch_bounds__(256) perplexity_kernel(int N, int S, const int32_t* __restrict__ seg,
+                                                        const float* __restrict__ s_sum,
+                                                        const float* __restrict__ t_sum,
+                                                        const int32_t* __restrict__ count,
+                                                        float* ppl_s, float* ppl_t) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= N) return;
+  const int c = seg[i];
+  const float nan = __int_as_float(0x7fc00000);
+  float ps = nan, pt = nan;
+  if (c >= 0 && c < S && count[c] > 0) {
+    const float n = static_cast<float>(count[c]);
+    if (s_sum != nullptr) ps = expf(__fdiv_rn(s_sum[c], n));
+    if (t_sum != nullptr) pt = expf(__fdiv_rn(t_sum[c], n));
+  }
+  if (ppl_s != nullptr) ppl_s[i] = ps;
+  if (ppl_t != nullptr) ppl_t[i] = pt;
+}
+
+// Self-test of the bounded-wait path, on a healthy device: one CTA of 128 threads waits, with the
+// same mbar_wait the tensor kernels use, on an mbarrier that nothing ever arrives on.  When the
+// (short) limit runs out the threads agree to leave through the same vote barrier the epilogue
+// groups use, and the status word receives the time-out code the same way the tensor kernels
+// report it.  No copy and no MMA is in flight; the kernel always terminates.
+//   out[0] = status word (must be 0 on entry), out[1] = 1 if every thread's wait returned false,
+//   out[2] = SM clock cycles thread 0 spent in the wait (low 31 bits)
+__global__ void __launch_bounds__(128) wait_timeout_selftest_kernel(long long limit_cycles, int* out) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  const long long t0 = clock64();
+  const bool okw = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar), 0, &abort_flag, limit_cycles));
+  const long long dt = clock64() - t0;
+  const bool ok = named_barrier_vote(1, 128, okw);
+  const int none_ok = __syncthreads_and(okw ? 0 : 1);
+  if (threadIdx.x == 0) {
+    if (!ok && abort_flag != 0) atomicCAS(out, 0, kStatusTimeout);
+    out[1] = none_ok;
+    out[2] = static_cast<int>(dt & 0x7fffffff);
+  }
+}
+
 // fp32 dH accumulator over the compact rows -> bf16 [T, ld] output by token; tokens without a
 // compact row (no loss) get zeros.  8 elements per thread.
 __global__ void __launch_bounds__(256) scatter_dhidden_kernel(const float* __restrict__ src,

@@ -527,3 +527,58 @@ def test_host_buffer_entry_point_matches_device_entry_point():
         B.npd_kd_fwd_bwd_host_streams(hargs, step.args, copy_stream, compute)
     torch.cuda.synchronize()
     assert torch.equal(hkl, ref.kl.cpu()) and torch.equal(step.d_weight, ref.d_weight)
+
+
+def test_perplexity_scores_match_the_oracle():
+    b = syn.config4_short(device=DEV, T=2048, d=128, V=3000)
+    step = run_step(b, grads=False)
+    kl, ns, nt = check_full_parity(b, step, check_grads=False)
+    cu, y, m = b.cu_seqlens.cpu().numpy(), b.labels.cpu().numpy(), b.loss_mask.cpu().numpy()
+    ref = orc.segment_stats(cu, m, y, kl, ns, nt)
+    got = B.npd_segment_stats(b.cu_seqlens, b.loss_mask, b.labels, step.kl, step.nll_student, step.nll_teacher)
+    seg = torch.arange(b.S, dtype=torch.int32, device=DEV)
+    ps, pt = B.npd_perplexity(seg, got[1], got[2], got[3])
+    torch.cuda.synchronize()
+    assert_losses_close(host(ps), orc.perplexity_scores(np.arange(b.S), ref[1], ref[3]), "ppl_student")
+    assert_losses_close(host(pt), orc.perplexity_scores(np.arange(b.S), ref[2], ref[3]), "ppl_teacher")
+    # the same two operations in float32 on the same sums: bit for bit up to the exponential's last place
+    o32 = orc.perplexity_scores(np.arange(b.S), host(got[1]), got[3].cpu().numpy(), dtype=np.float32)
+    assert np.allclose(host(ps), o32, rtol=3e-7, atol=0, equal_nan=True)
+    # empty sample and a segment index out of range: NaN; one output alone is allowed
+    cnt = got[3].clone()
+    cnt[1] = 0
+    bad = torch.tensor([1, -1, b.S, 0], dtype=torch.int32, device=DEV)
+    ps2, none = B.npd_perplexity(bad, got[1], None, cnt)
+    assert none is None
+    p = host(ps2)
+    assert np.isnan(p[:3]).all() and np.isfinite(p[3])
+    with pytest.raises(B.NpdError):
+        B.npd_perplexity(bad, None, None, cnt)
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    # a wait on a barrier nothing arrives on, with a limit of 2e5 cycles (about 0.1 ms): the status
+    # word must read NPD_ETIMEOUT, every thread must have given up, and the device must be fine
+    import time
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    out = B.npd_selftest_wait_timeout(200_000, device=DEV)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    status, all_gave_up, cycles = out.cpu().tolist()
+    assert status == B.NPD_ETIMEOUT and all_gave_up == 1
+    assert 200_000 <= cycles < 1_000_000
+    assert dt < 0.5
+    with pytest.raises(B.NpdError):
+        B.npd_selftest_wait_timeout(10**9, device=DEV)          # refused on the host: too long
+    # the context is still usable
+    b = syn.config1_tiny(device=DEV, teacher_dtype=torch.bfloat16)
+    check_full_parity(b, run_step(b))
+
+
+def test_serialized_launches_give_the_same_results():
+    b = syn.config2_1b(device=DEV, T=1024, d=256, V=5000, min_len=32, max_len=256)
+    s1 = run_step(b, grad_chunk_cols=1024)
+    s2 = run_step(b, grad_chunk_cols=1024, flags=B.NPD_KD_SERIALIZE_LAUNCHES)
+    assert torch.equal(s1.kl, s2.kl) and torch.equal(s1.d_weight, s2.d_weight)
+    assert frob(host(s1.d_hidden), host(s2.d_hidden)) < 1e-3
