@@ -71,11 +71,7 @@ def lib() -> C.CDLL:
     if _lib is None:
         from . import build as _build
         if _build.is_stale():          # missing, or built from other sources than the ones present
-            try:
-                _build.build()
-            except RuntimeError:
-                if not os.path.exists(LIB_PATH):
-                    raise
+            _build.build()             # raises if it cannot: never run kernels of other sources
         if not os.path.exists(LIB_PATH):
             raise RuntimeError(
                 f"{LIB_PATH} is missing: build it with `python -m paper_2605_05940_b200.build` "
@@ -353,26 +349,39 @@ class KDStep:
     def run(self, stream=None):
         npd_kd_fwd_bwd(self.args, stream)
 
-    def run_with_phase_times(self, stream=None):
-        """One step with the library's phase events attached.  Returns a list of
-        (group name, milliseconds); synchronises."""
+    def phase_names(self):
+        """Names of the launch groups of a call, in the order their phase events are recorded."""
         groups, chunks = npd_phase_count(self.args)
         names = ["forward_tiles", "merge"]
         for _ in range(chunks):
             names += ["gradient_tiles", "backward_gemms"]
         names += ["dhidden_convert"] * (groups - len(names))
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(groups + 1)]
-        # an event only owns a CUDA handle once it has been recorded
+        return names
+
+    def new_phase_events(self, stream=None):
+        """groups + 1 timing events, each recorded once so that it owns a CUDA handle."""
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(self.phase_names()) + 1)]
         s = torch.cuda.current_stream() if stream is None else stream
         for e in evs:
             e.record(s)
+        return evs
+
+    def run_recording(self, evs, stream=None):
+        """One step with the library's phase events attached; only enqueues."""
         arr = (C.c_void_p * len(evs))(*[e.cuda_event for e in evs])
         a = npd_kd_args.from_buffer_copy(self.args)
         a.phase_events = C.cast(arr, C.POINTER(C.c_void_p))
         a.n_phase_events = len(evs)
         npd_kd_fwd_bwd(a, stream)
+
+    def run_with_phase_times(self, stream=None):
+        """One step with the library's phase events attached.  Returns a list of
+        (group name, milliseconds); synchronises."""
+        names = self.phase_names()
+        evs = self.new_phase_events(stream)
+        self.run_recording(evs, stream)
         torch.cuda.synchronize()
-        return [(names[i], evs[i].elapsed_time(evs[i + 1])) for i in range(groups)]
+        return [(names[i], evs[i].elapsed_time(evs[i + 1])) for i in range(len(names))]
 
     def status(self, stream=None) -> int:
         return npd_last_status(self._ws_view, stream)

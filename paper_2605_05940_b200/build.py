@@ -47,8 +47,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
     """Compile libnpd.so for sm_100a if it is missing or older than its sources."""
     if not force and not is_stale():
         return LIB_PATH
+    # nvcc writes to a name of its own and the finished file is moved into place, so that a
+    # process loading the library at the same moment never sees half of it
+    tmp = f"{LIB_PATH}.{os.getpid()}.tmp"
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3",
-           "-std=c++17", "-shared", "-Xcompiler", "-fPIC", "-o", LIB_PATH] + SOURCES
+           "-std=c++17", "-shared", "-Xcompiler", "-fPIC", "-o", tmp] + SOURCES
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
@@ -56,9 +59,15 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if verbose:
         sys.stderr.write(res.stderr)
     if res.returncode != 0:
+        if os.path.exists(tmp):
+            os.remove(tmp)
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-    with open(STAMP_PATH, "w") as f:
+    if os.path.exists(STAMP_PATH):
+        os.remove(STAMP_PATH)          # no stamp while the library and the stamp could disagree
+    os.replace(tmp, LIB_PATH)
+    with open(STAMP_PATH + ".tmp", "w") as f:
         f.write(sources_digest() + "\n")
+    os.replace(STAMP_PATH + ".tmp", STAMP_PATH)
     return LIB_PATH
 
 

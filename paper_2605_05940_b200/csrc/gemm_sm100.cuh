@@ -29,11 +29,15 @@
 // the drain of a tile is not overlapped with the next tile's MMAs (a few per cent at the
 // k-extents used here).
 //
-// One CTA per SM, 320 threads: warp 0 = TMA producer, warp 1 = TMEM owner and, in the leader
+// One CTA per SM, 384 threads: warp 0 = TMA producer, warp 1 = TMEM owner and, in the leader
 // CTA (cluster rank 0), the MMA issuer of the pair, warps 2-9 = epilogue in two groups of
-// four warps (one accumulator row per thread, each group drains half of the columns):
-// TMEM -> registers -> 128-byte-swizzled shared memory -> TMA store, or TMA reduce-add for
-// outputs that are accumulated (split-K, or several launches adding into one matrix).
+// four warps (one accumulator row per thread, each group drains half of the columns), warps
+// 10 and 11 = one storing thread per group.  An accumulator leaves through a ring of two small
+// staging buffers per group: TMEM -> registers -> 64-byte-swizzled shared memory (128 rows x
+// 64 bytes) -> TMA store, or TMA reduce-add for outputs that are accumulated (split-K, the
+// stream-K pieces, several launches adding into one matrix).  The epilogue warps fill a buffer and
+// signal it; the storing thread issues the copy and frees the buffer when the copy has read it,
+// with one copy in flight while the next buffer is filled.  All roles meet at mbarriers only.
 #pragma once
 
 #include "ptx_sm100.cuh"
@@ -71,13 +75,14 @@ constexpr int BK = 64, UK = 16, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;             // 16 KB
 constexpr int BSUB_BYTES = (BNS / 2) * BK * 2;   // 16 KB: this CTA's half of one 256-row block of B
 constexpr int B_BYTES = NSUB * BSUB_BYTES;       // 32 KB
-constexpr int OUT_BYTES = 128 * 128;             // staging of one epilogue group: 128 rows x 128 B
-constexpr int THREADS = 320;
+constexpr int OUT_BYTES = 128 * 64;              // one staging buffer: 128 rows x 64 B
+constexpr int OUT_BUFS = 2;                      // staging buffers per epilogue group
+constexpr int THREADS = 384;
 constexpr int TMEM_COLS = 512;
 constexpr int OFF_A = 0;
 constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
 constexpr int OFF_OUT = OFF_B + STAGES * B_BYTES;
-constexpr int OFF_BAR = OFF_OUT + 2 * OUT_BYTES;
+constexpr int OFF_BAR = OFF_OUT + 2 * OUT_BUFS * OUT_BYTES;
 constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;  // + barriers + alignment
 }  // namespace gemm_cfg
 
@@ -249,8 +254,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
   uint8_t* smem_a = smem + OFF_A;
   uint8_t* smem_b = smem + OFF_B;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + OFF_BAR);
-  // bars[0..S) full, [S..2S) empty, [2S] tmem full, [2S+1] tmem empty
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2);
+  // bars[0..S) full, [S..2S) empty, [2S] tmem full, [2S+1] tmem empty,
+  // [2S+2 ..) staging buffer filled [group][buffer], then staging buffer free [group][buffer]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2 + 4 * OUT_BUFS);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5;
@@ -260,6 +266,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
   const int num_clusters = gridDim.x >> 1;
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + STAGES);
   const uint32_t tfull = smem_u32(bars + 2 * STAGES), tempty = smem_u32(bars + 2 * STAGES + 1);
+  const uint32_t ofull0 = smem_u32(bars + 2 * STAGES + 2), oempty0 = ofull0 + 8 * 2 * OUT_BUFS;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -268,6 +275,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
     }
     mbar_init(tfull, 1);
     mbar_init(tempty, 16);  // 8 epilogue warps of each CTA, counted in the leader
+    for (int i = 0; i < 2 * OUT_BUFS; ++i) {
+      mbar_init(ofull0 + 8 * i, 4);   // the four warps of the group
+      mbar_init(oempty0 + 8 * i, 1);  // the group's storing thread
+    }
     *abort_flag = 0;
     fence_mbar_init();
     prefetch_tmap(&tmap_a0);
@@ -395,86 +406,108 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmap_a0, const __grid_const
     }
   } else {
     // ------------------------------ epilogue ----------------------------------
-    const int e = warp - 2;
-    const int lg = warp & 3;   // TMEM lane group this warp may read
-    const int grp = e >> 2;    // epilogue group: which half of the tile's columns
-    const int row_local = lg * 32 + lane;
-    const uint32_t swz = static_cast<uint32_t>(row_local & 7);
-    uint8_t* obuf = smem + OFF_OUT + grp * OUT_BYTES;
-    uint8_t* orow = obuf + row_local * 128;
-    const bool issuer = (e & 3) == 0 && lane == 0;
-    const int bar_id = 1 + grp;
-    uint32_t tile = 0;
+    // What a group does with one unit, the same for its four warps and its storing thread:
+    // sub-tiles of 64 output bytes per row (16 fp32 or 32 bf16 columns), `nsteps` of them.
+    const bool storer = warp >= 10;
+    const int grp = storer ? warp - 10 : (warp - 2) >> 2;  // which half of the tile's columns
+    auto unit_steps = [&](const GemmProblem& g, const GemmUnit& u, int& c0, int& step) {
+      const int gcols = (BNS / 2) * u.ns;         // accumulator columns this group drains
+      c0 = grp * gcols;                           // the first of them
+      step = g.out_f32 ? 16 : 32;
+      const int m0 = u.m0 + static_cast<int>(rank) * BM;
+      if (m0 >= g.M) return 0;                    // this CTA's 128 rows lie beyond M: nothing to store
+      int n = (g.N - (u.n0 + c0) + step - 1) / step;  // sub-tiles of this group that lie inside N
+      return n < 0 ? 0 : (n > gcols / step ? gcols / step : n);
+    };
+    uint32_t oit = 0;  // staging buffers used so far by this group (same count in all five roles)
     bool ok = true;
     int prob;
     GemmUnit u;
-    for (; ok && walk.next(prob, u); ++tile) {
-      const GemmProblem& g = prob ? walk.pr[1] : walk.pr[0];
-      const CUtensorMap* to = prob ? &tmap_o1 : &tmap_o0;
-      const int m0 = u.m0 + static_cast<int>(rank) * BM;
-      const bool rows_inside = m0 < g.M;          // else this CTA's 128 rows lie beyond M: nothing to store
-      const int out_row0 = m0;
-      const bool no_k = u.kt0 == u.kt1;           // empty k range: the accumulators hold nothing, D = 0
-      const int gcols = (BNS / 2) * u.ns;         // accumulator columns this group drains
-      const int c0 = grp * gcols;                 // the first of them
-      const int step = g.out_f32 ? 32 : 64;       // columns per staged sub-tile (128 bytes of output)
-      // sub-tiles of this group that lie inside N (uniform over the group)
-      int nsteps = (g.N - (u.n0 + c0) + step - 1) / step;
-      nsteps = nsteps < 0 ? 0 : (nsteps > gcols / step ? gcols / step : nsteps);
-      // the four warps of a group stay or leave together (they meet at barriers below)
-      ok = named_barrier_vote(bar_id, 128, __all_sync(0xffffffffu, mbar_wait(tfull, tile & 1, abort_flag)));
-      if (!ok) break;
-      tc_fence_after_sync();
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + c0;
-      if (nsteps == 0) {
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive_cluster(tempty_leader);
-      }
-      for (int j = 0; j < nsteps; ++j) {
-        uint32_t w[32];  // 128 bytes of this thread's output row
-        if (no_k) {
-#pragma unroll
-          for (int q = 0; q < 32; ++q) w[q] = 0u;
-        } else if (g.out_f32) {
-          tmem_ld32(taddr + j * 32, w);
-          tmem_ld_wait();
-        } else {
-          uint32_t r0[32], r1[32];
-          tmem_ld32(taddr + j * 64, r0);
-          tmem_ld32(taddr + j * 64 + 32, r1);
-          tmem_ld_wait();
-#pragma unroll
-          for (int q = 0; q < 16; ++q) {
-            w[q] = pack_bf16x2(__uint_as_float(r0[2 * q]), __uint_as_float(r0[2 * q + 1]));
-            w[16 + q] = pack_bf16x2(__uint_as_float(r1[2 * q]), __uint_as_float(r1[2 * q + 1]));
+    if (storer) {
+      if (lane == 0) {
+        int prev = -1;  // buffer of the copy in flight
+        while (ok && walk.next(prob, u)) {
+          const GemmProblem& g = prob ? walk.pr[1] : walk.pr[0];
+          const CUtensorMap* to = prob ? &tmap_o1 : &tmap_o0;
+          int c0, step;
+          const int nsteps = unit_steps(g, u, c0, step);
+          const int row0 = u.m0 + static_cast<int>(rank) * BM;
+          for (int j = 0; j < nsteps; ++j, ++oit) {
+            const int b = grp * OUT_BUFS + static_cast<int>(oit % OUT_BUFS);
+            if (!(ok = mbar_wait(ofull0 + 8 * b, (oit / OUT_BUFS) & 1, abort_flag))) break;
+            const uint32_t src = smem_u32(smem + OFF_OUT + b * OUT_BYTES);
+            const int col = u.n0 + c0 + j * step;
+            if (g.out_reduce)
+              tma_reduce_add_2d(to, src, col, row0);
+            else
+              tma_store_2d(to, src, col, row0);
+            tma_store_commit();
+            if (prev >= 0) {
+              tma_store_wait_read<1>();  // the copy before this one has read its buffer
+              mbar_arrive(oempty0 + 8 * prev);
+            }
+            prev = b;
           }
         }
-        if (j == nsteps - 1) {
-          // everything this warp needs from tensor memory is in registers: release the accumulators
+        tma_store_wait_read<0>();
+        if (prev >= 0) mbar_arrive(oempty0 + 8 * prev);
+        tma_store_wait_all<0>();
+      }
+    } else {
+      const int lg = warp & 3;   // TMEM lane group this warp may read
+      const int row_local = lg * 32 + lane;
+      const uint32_t swz = static_cast<uint32_t>((row_local >> 1) & 3);  // 64-byte swizzle
+      uint32_t tile = 0;
+      for (; ok && walk.next(prob, u); ++tile) {
+        const GemmProblem& g = prob ? walk.pr[1] : walk.pr[0];
+        const bool no_k = u.kt0 == u.kt1;           // empty k range: the accumulators hold nothing, D = 0
+        int c0, step;
+        const int nsteps = unit_steps(g, u, c0, step);
+        ok = __all_sync(0xffffffffu, mbar_wait(tfull, tile & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + c0;
+        if (nsteps == 0) {
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(tempty_leader);
         }
+        for (int j = 0; j < nsteps; ++j, ++oit) {
+          uint32_t w[16];  // 64 bytes of this thread's output row
+          if (no_k) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
-          *reinterpret_cast<uint4*>(orow + ((static_cast<uint32_t>(q) ^ swz) << 4)) =
-              make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
-        fence_proxy_async_smem();
-        named_barrier_sync(bar_id, 128);
-        if (issuer && rows_inside) {
-          const int col = u.n0 + c0 + j * step;
-          if (g.out_reduce)
-            tma_reduce_add_2d(to, smem_u32(obuf), col, out_row0);
-          else
-            tma_store_2d(to, smem_u32(obuf), col, out_row0);
-          tma_store_commit();
-          tma_store_wait_read<0>();  // the staging buffer may be overwritten after this
+            for (int q = 0; q < 16; ++q) w[q] = 0u;
+          } else if (g.out_f32) {
+            tmem_ld16(taddr + j * 16, w);
+            tmem_ld_wait();
+          } else {
+            uint32_t r0[32];
+            tmem_ld32(taddr + j * 32, r0);
+            tmem_ld_wait();
+#pragma unroll
+            for (int q = 0; q < 16; ++q)
+              w[q] = pack_bf16x2(__uint_as_float(r0[2 * q]), __uint_as_float(r0[2 * q + 1]));
+          }
+          if (j == nsteps - 1) {
+            // everything this warp needs from tensor memory is in registers: release the accumulators
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(tempty_leader);
+          }
+          const int b = grp * OUT_BUFS + static_cast<int>(oit % OUT_BUFS);
+          ok = __all_sync(0xffffffffu, mbar_wait(oempty0 + 8 * b, ((oit / OUT_BUFS) & 1) ^ 1, abort_flag));
+          if (!ok) break;
+          uint8_t* orow = smem + OFF_OUT + b * OUT_BYTES + row_local * 64;
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4*>(orow + ((static_cast<uint32_t>(q) ^ swz) << 4)) =
+                make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(ofull0 + 8 * b);
         }
-        named_barrier_sync(bar_id, 128);
       }
     }
-    if (issuer) tma_store_wait_all<0>();
   }
 
   // ------------------------------ teardown ------------------------------------

@@ -31,8 +31,13 @@
 //               In both CTAs this warp owns the 512 TMEM columns (2 accumulators 128x256).
 //   warp 2      TMA producer for this CTA's teacher sub-tiles (a ring of 2 or 3 stages per column half); the rows of a
 //               block lie anywhere in the packed batch, so each lane gathers four of them
+//   warp 3      gradient pass only: one thread hands each finished gradient sub-tile to a TMA
+//               store and recycles the stage when the store has read it
 //   warps 4-11  epilogue; warp w reads TMEM lanes 32*(w%4).., columns 128*((w-4)/4)..
 //               so every thread owns one token row and half of the tile's columns.
+// The roles only ever meet at mbarriers (every wait on one is bounded), with one exception: with
+// an fp32 teacher the four epilogue warps of a column half pass a named barrier before they
+// overwrite the teacher sub-tile; that barrier carries a vote so that they leave together.
 // All exponentials are taken in base 2 on logits pre-scaled by log2(e)/tau.
 //
 // kSparse: the teacher is given as its k largest logits per token (Eq. 2 as printed) instead
@@ -114,7 +119,7 @@ struct Layout {
   static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
   static constexpr int OFF_Z = OFF_B + STAGES * B_BYTES;
   static constexpr int OFF_BAR = OFF_Z + 2 * ZQ * ZSUB_BYTES;
-  static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * ZQ;
+  static constexpr int NUM_BARS = 2 * STAGES + 4 + 6 * ZQ;
   static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;
 };
 // Teacher logits are clamped below at this value: a finite stand-in for the -inf entries of
@@ -153,6 +158,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
   const uint32_t tempty0 = tfull0 + 16;
   const uint32_t zfull0 = tempty0 + 16;           // [half][ZQ]
   const uint32_t zempty0 = zfull0 + 8 * 2 * ZQ;   // [half][ZQ]
+  const uint32_t gfull0 = zempty0 + 8 * 2 * ZQ;   // [half][ZQ] gradient sub-tile written (gradient pass)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
@@ -165,7 +171,10 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
     }
     for (int i = 0; i < 2 * ZQ; ++i) {
       mbar_init(zfull0 + 8 * i, 1);
+      // a stage is given back by the four epilogue warps of its half (forward pass) or by the
+      // thread that stores the gradient sub-tile once the store has read it (gradient pass)
       mbar_init(zempty0 + 8 * i, kMode == kForward ? 4 : 1);
+      mbar_init(gfull0 + 8 * i, 4);
     }
     *abort_flag = 0;
     fence_mbar_init();
@@ -322,6 +331,37 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           mbar_wait_drain(zfull0 + 8 * (half * ZQ + (i2 % ZQ)), (i2 / ZQ) & 1);
       }
     }
+  } else if (warp == 3) {
+    // ---------------------- gradient sub-tile store (gradient pass) ----------------------
+    // One thread hands every finished 128 x 64 gradient sub-tile to TMA and, once the store has
+    // read it, gives the stage back (to the teacher producer, or with a top-k teacher to the
+    // epilogue warps).  The epilogue warps never wait for a store.
+    if (kMode == kGradient && lane == 0) {
+      uint32_t zit = 0;
+      bool ok = true;
+      for (int u = cluster_id; u < units && ok; u += num_clusters) {
+        int slot, r, s, vt0, vt1;
+        run_of(u, slot, r, s, vt0, vt1);
+        for (int vt = vt0; vt < vt1 && ok; ++vt) {
+          for (int j = 0; j < BN / 2 / ZC && ok; ++j, ++zit) {
+            const uint32_t q = zit % ZQ, ph = (zit / ZQ) & 1;
+            for (int half = 0; half < 2 && ok; ++half) {
+              const uint32_t bi = 8 * (half * ZQ + q);
+              if (!(ok = mbar_wait(gfull0 + bi, ph, abort_flag))) break;
+              if (r >= 0)
+                tma_store_2d(&tmap_g, smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES),
+                             vt * BN + half * (BN / 2) + j * ZC - p.g_col0, r);
+            }
+            if (!ok) break;
+            tma_store_commit();
+            tma_store_wait_read<0>();
+            mbar_arrive(zempty0 + 8 * q);
+            mbar_arrive(zempty0 + 8 * (ZQ + q));
+          }
+        }
+      }
+      tma_store_wait_all<0>();
+    }
   } else if (warp >= 4) {
     // ---------------------- epilogue ----------------------
     const int e = warp - 4;
@@ -365,12 +405,13 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
       }
       for (int vt = vt0; vt < vt1 && ok; ++vt, ++tile) {
         const uint32_t buf = tile & 1, tph = (tile >> 1) & 1;
-        // okw: this warp's waits so far succeeded.  In the forward pass a warp that gives up just
-        // leaves.  In the gradient pass the four warps of a column half meet at named barriers, so
-        // a warp whose wait ran out keeps joining them (doing nothing else) until the vote at the
-        // end of the sub-tile tells the whole half to leave together.
+        // okw: this warp's waits so far succeeded.  A warp that gives up just leaves, except in the
+        // gradient pass with an fp32 teacher: there the four warps of a column half meet at a
+        // named barrier before they write, so a warp whose wait ran out still joins that barrier
+        // (doing nothing else), and the barrier's vote tells the whole half to leave together.
+        constexpr bool kMeets = kMode == kGradient && kTeacherF32;
         bool okw = __all_sync(0xffffffffu, mbar_wait(tfull0 + 8 * buf, tph, abort_flag));
-        if (kMode == kForward && !okw) { ok = false; break; }
+        if (!kMeets && !okw) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t taddr =
             tmem_base + (static_cast<uint32_t>(lg * 32) << 16) + buf * BN + half * (BN / 2);
@@ -379,9 +420,16 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           const uint32_t bi = 8 * (half * ZQ + q);
           if (!kSparse) {
             okw = okw && __all_sync(0xffffffffu, mbar_wait(zfull0 + bi, zph, abort_flag));
-            if (kMode == kForward && !okw) { ok = false; break; }
+          } else if (kMode == kGradient) {
+            // no teacher stream: the stage is free once the store of its last sub-tile has read it
+            okw = okw && __all_sync(0xffffffffu, mbar_wait(zempty0 + bi, zph ^ 1, abort_flag));
           }
-          if (kMode == kGradient && kTeacherF32 && !okw) named_barrier_sync(1 + half, 128);  // see below
+          if (!kMeets && !okw) { ok = false; break; }
+          if (kMeets && !okw) {   // stands in for the barrier inside the loop below
+            named_barrier_vote(1 + half, 128, false);
+            ok = false;
+            break;
+          }
           uint8_t* zrow = smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES + row_local * 128;
           const int sub_col0 = vt * BN + half * (BN / 2) + j * ZC;
 #pragma unroll 1
@@ -514,7 +562,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
               if (kTeacherF32) {
                 // 64-byte gradient rows, dense from the start of the stage: they overlap other
                 // threads' teacher rows, so everyone of this half must have read its row first
-                named_barrier_sync(1 + half, 128);
+                if (!named_barrier_vote(1 + half, 128, true)) { ok = false; break; }
                 uint8_t* grow = smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES + row_local * 64;
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
@@ -534,23 +582,11 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
               if (lane == 0) mbar_arrive(zempty0 + bi);
             }
           } else {
-            // hand the finished 128 x 64 gradient sub-tile to TMA, then recycle the stage
-            fence_proxy_async_smem();
-            ok = named_barrier_vote(1 + half, 128, okw);
+            // this warp's 32 rows of the gradient sub-tile are written: tell the storing thread
             if (!ok) break;
-            if (lg == 0 && lane == 0) {
-              if (r >= 0) {
-                tma_store_2d(&tmap_g, smem_u32(smem + OFF_Z + (half * ZQ + q) * ZSUB_BYTES),
-                             sub_col0 - p.g_col0, r);
-                tma_store_commit();
-                tma_store_wait_read<0>();
-              }
-              // dense teacher: the stage goes back to the teacher producer.  Top-k teacher: the
-              // two stages of a half simply alternate; this thread has seen the store's read
-              // finish before it joins the next sub-tile's barrier, which every writer of the
-              // sub-tile after that has to pass first.
-              if (!kSparse) mbar_arrive(zempty0 + bi);
-            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(gfull0 + bi);
           }
         }
         if (!ok) break;
@@ -571,7 +607,6 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         }
       }
     }
-    if (kMode == kGradient && lg == 0 && lane == 0) tma_store_wait_all<0>();
   }
 
   // ---------------------- teardown ----------------------

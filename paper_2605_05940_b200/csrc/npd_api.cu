@@ -40,10 +40,12 @@ PFN_cuTensorMapEncodeTiled_v12000 tensor_map_encoder() {
   return fn;
 }
 
-// 2-D tensor map with 128-byte swizzle.  inner = contiguous extent (elements), outer = rows,
-// ld = row stride (elements), box = {box_inner (128 bytes' worth), box_outer}.
+// 2-D tensor map, 128-byte swizzle by default (swizzle64: 64-byte swizzle for boxes with 64-byte
+// rows).  inner = contiguous extent (elements), outer = rows, ld = row stride (elements),
+// box = {box_inner, box_outer}.
 bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, uint64_t ld,
-              uint32_t box_inner, uint32_t box_outer, bool f32 = false, bool swizzle = true) {
+              uint32_t box_inner, uint32_t box_outer, bool f32 = false, bool swizzle = true,
+              bool swizzle64 = false) {
   auto enc = tensor_map_encoder();
   if (enc == nullptr) return false;
   cuuint64_t dims[2] = {inner, outer};
@@ -52,7 +54,8 @@ bool make_map(CUtensorMap* m, const void* base, uint64_t inner, uint64_t outer, 
   cuuint32_t estr[2] = {1, 1};
   return enc(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
              const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-             swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+             swizzle ? (swizzle64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B)
+                     : CU_TENSOR_MAP_SWIZZLE_NONE,
              CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -276,9 +279,9 @@ int launch_gemm(int nprob, const GemmProblem* pr, const GemmOperands* ops, const
                             : make_map(&maps[3 * i], ops[j].A, ak, am, ops[j].lda, 64, BM);
     const bool okb = g.b_mn ? make_map(&maps[3 * i + 1], ops[j].B, g.N, bk, ops[j].ldb, 64, 64)
                             : make_map(&maps[3 * i + 1], ops[j].B, bk, g.N, ops[j].ldb, 64, BNS / 2);
-    // output sub-tiles: 128 rows x 128 bytes
-    const bool oko = make_map(&maps[3 * i + 2], ops[j].out, g.N, om, ops[j].ldo, g.out_f32 ? 32 : 64, BM,
-                              g.out_f32 != 0);
+    // output sub-tiles: 128 rows x 64 bytes, 64-byte swizzle
+    const bool oko = make_map(&maps[3 * i + 2], ops[j].out, g.N, om, ops[j].ldo, g.out_f32 ? 16 : 32, BM,
+                              g.out_f32 != 0, true, true);
     if (!oka || !okb || !oko) return NPD_ECUDA;
     gp.pr[i] = g;
     if (i < nprob)
