@@ -359,7 +359,8 @@ int npd_last_copy_bytes(int64_t* h2d_bytes, int64_t* d2h_bytes);
  * cudaFree or other allocating call.
  *
  * The first call on each device looks up the array's device address (with that device
- * current) and caches it; make that first call outside any stream capture.  All calls on
+ * current) and caches it; make that first call outside any stream capture.  The cached address
+ * does not survive a cudaDeviceReset of that device: do not use this entry point after one.  All calls on
  * a device share the one array and it keeps the previous call's contents: the library
  * clears the status word at the start of every call and overwrites every partial before
  * reading it, but two calls whose kernels overlap on the GPU (different streams, or

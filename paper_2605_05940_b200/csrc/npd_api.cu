@@ -1,6 +1,9 @@
 // Host side of the C ABI declared in include/npd.h: argument checks, workspace
 // layout, TMA descriptors and kernel launches.  Nothing here allocates device
-// memory or keeps state between calls.
+// memory, and no problem state survives a call.  What does persist: two per-thread diagnostic
+// counters, the per-device list of kernels whose shared-memory limit has been raised, and, for
+// npd_kd_forward_noalloc alone, a fixed scratch array in the library image with its cached
+// per-device address (which does not survive a cudaDeviceReset).
 #include "../../include/npd.h"
 
 #include <cuda.h>
