@@ -1,15 +1,22 @@
 #!/usr/bin/env python
 """Benchmark of the fused packed KD forward+backward step (one JSON line).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config c2|c3|c4|c5]
 
-A step is one pass of the whole hot path over one synthetic batch of the ~1B-student
-workload (T=8192 packed tokens, d=1536, V=151,936, bf16, tau=1): LM-head tiles with
+A step is one pass of the whole hot path over one synthetic batch: LM-head tiles with
 online softmax, per-token merge, gradient tiles, dW and dH contractions, then the
-segment reductions and the Delta-IFD selection.  `value` is packed tokens/s with the
+segment reductions and the Delta-IFD selection.  The default workload is the ~1B-student
+shape the metric is quoted on (c2: T=8192 packed tokens, d=1536, V=151,936, bf16, tau=1);
+--config picks one of the other full-size shapes.  `value` is packed tokens/s with the
 inputs resident in HBM; `e2e` is the same step through the host-buffer entry point
 (host->device copies of hidden states, teacher logits, boundaries, mask and labels and
 the device->host read of the per-token losses inside the timed region).
+
+After the timed loop the same loop runs once more with the library's phase events
+attached, clocks sampled: `roofline` is the dominant launch group as timed there (so
+its time is part of a sustained step, not of a cold single launch), `phase_ms` /
+`phase_mcycles` / `tensor_pipe_frac_at_loop_clock` give every group's time, SM cycles
+and tensor-pipe utilisation at the clock the loop ran at.
 
 With N > 1 (launched under torch.distributed.run) every rank runs an independent
 replica on its own GPU - the path has no collective - and `value` is the sum over
@@ -53,10 +60,10 @@ UNIT = "tokens/s"
 # capture of dram__bytes_read.sum + dram__bytes_write.sum at full size.  They describe the kernels
 # as they were when the counters were taken: the digest is of the kernel sources at that time,
 # and once a source file has changed the figure is no longer reported.
-TRAFFIC = {"csrc_sha256_16": "none yet",
-           "forward_tiles": None,
-           "gradient_tiles": None,
-           "backward_gemms": None}
+TRAFFIC = {"csrc_sha256_16": "a3aa269f11b17055",
+           "forward_tiles": 2_367_577_344 + 7_972_352,
+           "gradient_tiles": 248_713_472 + 145_788_416,
+           "backward_gemms": 674_204_672 + 82_762_240}
 
 
 def _csrc_digest():
@@ -483,7 +490,7 @@ def run_ours(args):
                      "achieved": achieved if consistent else None, "peak": peak_tf,
                      "unit": "TFLOP/s", "frac": achieved / peak_tf if consistent else None,
                      "frac_of_burst_peak": achieved / peaks["bf16"] if consistent else None,
-                     "traffic": (traffic / launches_dom) if traffic else None,
+                     "traffic": traffic,
                      "traffic_note": "DRAM bytes per launch (ncu, full size); launches per step: %d" % launches_dom,
                      "peak_source": f"{peaks['source']} cuBLAS bf16, sustained (kernel timed inside the loop)",
                      "kernel_ms_per_step": dom_ms, "kernel_flops_per_step": dom_flops,
