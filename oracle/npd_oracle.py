@@ -58,6 +58,7 @@ __all__ = [
     "topk_kd_token_losses",
     "topk_kd_logit_gradient",
     "topk_kd_backward",
+    "validate_step_inputs",
     "validate_cu_seqlens",
     "segment_ids",
     "segment_stats",
@@ -316,6 +317,30 @@ def topk_kd_backward(H, W, topk_values, topk_indices, loss_mask, tau: float, gra
 # --------------------------------------------------------------------------- #
 # Packed segments (sequence packing, Algorithm 1 Phase 1) and their statistics
 # --------------------------------------------------------------------------- #
+
+def validate_step_inputs(H, teacher_logits, labels, loss_mask, V: int, topk_indices=None) -> bool:
+    """What the step may assume about its inputs and does not check by default.  True iff
+      * every label is below V (a label < 0 means "none"; one >= V names no class),
+      * with a dense teacher: no logit of a token that carries loss is NaN or +inf, and every such
+        token has at least one finite teacher logit (-inf entries only remove classes from the support
+        of Eq. 2; a row that is entirely -inf has no distribution),
+      * with a top-k teacher: every stored index lies in [0, V),
+      * the hidden states of the tokens that carry loss are finite.
+    Tokens with loss_mask 0 are never read by the step, so nothing is required of their rows."""
+    m = np.asarray(loss_mask).astype(bool)
+    y = np.asarray(labels, dtype=np.int64)
+    if np.any(y >= V):
+        return False
+    if not np.all(np.isfinite(_f64(H)[m])):
+        return False
+    if topk_indices is not None:
+        idx = np.asarray(topk_indices, dtype=np.int64)[m]
+        return bool(np.all((idx >= 0) & (idx < V)))
+    Z = _f64(teacher_logits)[m][:, :V]
+    if np.any(np.isnan(Z)) or np.any(np.isposinf(Z)):
+        return False
+    return bool(np.all(np.any(np.isfinite(Z), axis=1)))
+
 
 def validate_cu_seqlens(cu, T: int) -> bool:
     """True iff cu is a valid boundary list: cu[0]=0, strictly increasing,

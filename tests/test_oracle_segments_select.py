@@ -346,3 +346,38 @@ def test_perplexity_of_a_uniform_model_is_the_vocabulary_size():
     _, s_sum, t_sum, cnt = orc.segment_stats([0, 2, 6], m, y, kl, ns, nt)
     assert np.allclose(orc.perplexity_scores([0, 1], s_sum, cnt), V, rtol=1e-12)
     assert np.allclose(orc.perplexity_scores([0, 1], t_sum, cnt), V, rtol=1e-12)
+
+
+# --------------------------------------------------------------------------- #
+# Input validation (what the debug mode of the step checks)
+# --------------------------------------------------------------------------- #
+
+def test_validate_step_inputs_literal_cases():
+    V = 6
+    H = np.ones((4, 3))
+    Z = np.zeros((4, V))
+    y = np.asarray([0, 5, -100, 2])
+    m = np.asarray([1, 1, 0, 1], dtype=np.uint8)
+    ok = lambda **kw: orc.validate_step_inputs(kw.get("H", H), kw.get("Z", Z), kw.get("y", y), kw.get("m", m), V,
+                                               kw.get("idx"))
+    assert ok()
+    assert not ok(y=np.asarray([0, 6, -100, 2]))                 # a label that names no class
+    assert ok(y=np.asarray([0, 5, -7, 2]))                       # any negative label means "none"
+    Zi = Z.copy(); Zi[1, :] = -np.inf
+    assert not ok(Z=Zi)                                          # a loss token without any support
+    Zi = Z.copy(); Zi[1, :5] = -np.inf
+    assert ok(Z=Zi)                                              # one class left: fine
+    Zi = Z.copy(); Zi[2, :] = -np.inf
+    assert ok(Z=Zi)                                              # the masked token's row is never read
+    Zi = Z.copy(); Zi[0, 3] = np.nan
+    assert not ok(Z=Zi)
+    Zi = Z.copy(); Zi[3, 0] = np.inf
+    assert not ok(Z=Zi)
+    Hi = H.copy(); Hi[3, 1] = np.inf
+    assert not ok(H=Hi)
+    Hi = H.copy(); Hi[2, 1] = np.nan
+    assert ok(H=Hi)                                              # masked token again
+    idx = np.asarray([[0, 5], [1, 2], [9, 9], [3, 4]])
+    assert ok(idx=idx)                                           # row 2 is masked
+    assert not ok(idx=np.asarray([[0, 6], [1, 2], [0, 0], [3, 4]]))
+    assert not ok(idx=np.asarray([[0, 5], [-1, 2], [0, 0], [3, 4]]))
