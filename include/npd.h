@@ -70,7 +70,8 @@ typedef enum npd_status {
   NPD_EWORKSPACE = -6,  /* workspace NULL, misaligned or smaller than npd_workspace_bytes() */
   NPD_ECUDA = -7,       /* a CUDA runtime or driver call failed */
   NPD_ETIMEOUT = -8,    /* a bounded device-side wait expired (found on the device) */
-  NPD_EUNSUPPORTED = -9 /* a documented option that this build does not implement */
+  NPD_EUNSUPPORTED = -9,/* a documented option that this build does not implement */
+  NPD_EDATA = -10       /* NPD_KD_DEBUG_CHECKS found an input the step may not be given (found on the device) */
 } npd_status;
 
 enum { NPD_DTYPE_BF16 = 0, NPD_DTYPE_F32 = 1 };
@@ -91,6 +92,14 @@ enum {
                                p_G = Softmax(teacher[t]/tau), i.e. the divergence of the current
                                learner from the logits of the policy that generated the data, which
                                the paper's appendix tracks as policy lag.  Needs finite logits. */
+  NPD_KD_DEBUG_CHECKS = 16, /* before anything else, check on the device what the kernels otherwise take on
+                               trust and record NPD_EDATA in the status word if it does not hold: every
+                               label below V; for every token that carries loss finite hidden states,
+                               and either (dense teacher) no NaN or +inf logit and at least one finite
+                               one - a row that is entirely -inf has no distribution - or (top-k
+                               teacher) every stored index inside [0, V).  Rows of tokens without loss
+                               are not read.  The step runs all the same; with NPD_EDATA its outputs are
+                               undefined.  Costs one more pass over the teacher logits. */
   NPD_KD_SERIALIZE_LAUNCHES = 8 /* launch every kernel fully serialised.  By default the tensor-core
                                kernels of a call are chained as programmatic dependent launches:
                                the blocks of the next kernel are scheduled, and set up their
@@ -323,7 +332,7 @@ int npd_debug_chunk_schedule(int32_t row_blocks, int32_t d, int32_t chunk_cols, 
 
 /* Synchronises `cuda_stream`, then reads the device-side status word of a
  * workspace that npd_kd_fwd_bwd used into *host_status (HOST): NPD_OK,
- * NPD_ESEQ or NPD_ETIMEOUT.  Returns NPD_ECUDA if the stream itself failed. */
+ * NPD_ESEQ, NPD_ETIMEOUT or (debug checks) NPD_EDATA.  Returns NPD_ECUDA if the stream itself failed. */
 int npd_last_status(const void* workspace, void* cuda_stream, int32_t* host_status);
 
 /* HOST.  Static description of a status code. */

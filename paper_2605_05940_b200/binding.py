@@ -18,12 +18,13 @@ LIB_PATH = os.path.join(_HERE, "libnpd.so")
 
 NPD_OK = 0
 NPD_EINVAL, NPD_ESHAPE, NPD_EALIGN, NPD_ESEQ, NPD_EARCH = -1, -2, -3, -4, -5
-NPD_EWORKSPACE, NPD_ECUDA, NPD_ETIMEOUT, NPD_EUNSUPPORTED = -6, -7, -8, -9
+NPD_EWORKSPACE, NPD_ECUDA, NPD_ETIMEOUT, NPD_EUNSUPPORTED, NPD_EDATA = -6, -7, -8, -9, -10
 NPD_DTYPE_BF16, NPD_DTYPE_F32 = 0, 1
 NPD_KD_ACCUMULATE_DW = 1
 NPD_KD_COMPOSITE_LOSS = 2
 NPD_KD_REVERSE_KL = 4
 NPD_KD_SERIALIZE_LAUNCHES = 8
+NPD_KD_DEBUG_CHECKS = 16
 NPD_SELECT_TEACHER_IFD_LE_1 = 1
 NPD_SELECT_SCORE_IFD_TEACHER, NPD_SELECT_SCORE_IFD_STUDENT = 2, 4
 NPD_SELECT_LO_EXCLUSIVE, NPD_SELECT_HI_EXCLUSIVE = 8, 16

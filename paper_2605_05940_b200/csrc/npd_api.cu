@@ -341,6 +341,7 @@ const char* npd_strerror(int status) {
     case NPD_ECUDA: return "CUDA call failed";
     case NPD_ETIMEOUT: return "bounded device-side wait expired";
     case NPD_EUNSUPPORTED: return "option not implemented";
+    case NPD_EDATA: return "input data the step may not be given (debug checks)";
     default: return "unknown status";
   }
 }
@@ -419,6 +420,25 @@ int npd_kd_fwd_bwd(const npd_kd_args* a, void* cuda_stream) {
     segment_stats_kernel<<<(a->S + 3) / 4, 128, 0, st>>>(a->T, a->S, a->cu_seqlens, nullptr, nullptr,
                                                         nullptr, nullptr, nullptr, nullptr, nullptr,
                                                         nullptr, nullptr, nullptr, status);
+    ++g_launches;
+  }
+
+  if (a->flags & NPD_KD_DEBUG_CHECKS) {
+    ValidateParams vp{};
+    vp.T = a->T;
+    vp.d = a->d;
+    vp.V = a->V;
+    vp.topk = a->topk;
+    vp.hidden = static_cast<const __nv_bfloat16*>(a->hidden);
+    vp.ldh = a->ldh;
+    vp.teacher = sparse ? nullptr : a->teacher;
+    vp.teacher_f32 = tf32 ? 1 : 0;
+    vp.ldt = a->ldt;
+    vp.tk_idx = sparse ? a->topk_indices : nullptr;
+    vp.loss_mask = a->loss_mask;
+    vp.labels = a->labels;
+    vp.status = status;
+    validate_inputs_kernel<<<(a->T + 7) / 8, 256, 0, st>>>(vp);
     ++g_launches;
   }
 

@@ -471,6 +471,55 @@ __global__ void __launch_bounds__(256) perplexity_kernel(int N, int S, const int
   if (ppl_t != nullptr) ppl_t[i] = pt;
 }
 
+struct ValidateParams {
+  int T, d, V, topk;
+  const __nv_bfloat16* hidden;
+  long long ldh;
+  const void* teacher;   // dense bf16 / fp32 logits, or NULL with a top-k teacher
+  int teacher_f32;
+  long long ldt;
+  const int32_t* tk_idx; // [T, topk] or NULL
+  const uint8_t* loss_mask;
+  const int32_t* labels;
+  int* status;
+};
+constexpr int kStatusData = -10;
+
+// Debug mode of the step: one warp per token checks what the kernels otherwise take on trust.
+// Every label must be below V.  For a token that carries loss: finite hidden states; with a dense
+// teacher no NaN or +inf logit and at least one finite one (a row that is entirely -inf has no
+// distribution); with a top-k teacher every stored index inside [0, V).  Rows of tokens without
+// loss are not read.  The first violation found sets the status word.
+__global__ void __launch_bounds__(256) validate_inputs_kernel(const ValidateParams p) {
+  const int lane = threadIdx.x & 31;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (t >= p.T) return;
+  bool bad = false;
+  if (p.labels != nullptr && lane == 0) bad = p.labels[t] >= p.V;
+  const bool on = p.loss_mask == nullptr || p.loss_mask[t] != 0;
+  if (on) {
+    const __nv_bfloat16* h = p.hidden + static_cast<size_t>(t) * p.ldh;
+    for (int k = lane; k < p.d; k += 32) bad |= !isfinite(__bfloat162float(h[k]));
+    if (p.tk_idx != nullptr) {
+      for (int j = lane; j < p.topk; j += 32) {
+        const int c = p.tk_idx[static_cast<size_t>(t) * p.topk + j];
+        bad |= c < 0 || c >= p.V;
+      }
+    } else if (p.teacher != nullptr) {
+      bool support = false;
+      const size_t row = static_cast<size_t>(t) * p.ldt;
+      for (int c = lane; c < p.V; c += 32) {
+        const float z = p.teacher_f32 ? static_cast<const float*>(p.teacher)[row + c]
+                                      : __bfloat162float(static_cast<const __nv_bfloat16*>(p.teacher)[row + c]);
+        bad |= isnan(z) || (isinf(z) && z > 0.f);
+        support |= isfinite(z);
+      }
+      bad |= !__any_sync(0xffffffffu, support);
+    }
+  }
+  if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(p.status, 0, kStatusData);
+}
+
 // Self-test of the bounded-wait path, on a healthy device: one CTA of 128 threads waits, with the
 // same mbar_wait the tensor kernels use, on an mbarrier that nothing ever arrives on.  When the
 // (short) limit runs out the threads agree to leave through the same vote barrier the epilogue

@@ -582,3 +582,46 @@ def test_serialized_launches_give_the_same_results():
     s2 = run_step(b, grad_chunk_cols=1024, flags=B.NPD_KD_SERIALIZE_LAUNCHES)
     assert torch.equal(s1.kl, s2.kl) and torch.equal(s1.d_weight, s2.d_weight)
     assert frob(host(s1.d_hidden), host(s2.d_hidden)) < 1e-3
+
+
+def test_debug_checks_flag_inputs_the_step_may_not_be_given():
+    def fresh():
+        return syn.config2_1b(device=DEV, T=600, d=128, V=2000, min_len=20, max_len=200)
+
+    def status_of(b, **kw):
+        step = B.KDStep(b, flags=B.NPD_KD_DEBUG_CHECKS, **kw)
+        step.run()
+        torch.cuda.synchronize()
+        H, _, Z, y, m = oracle_inputs(b)
+        idx = kw["topk_indices"].cpu().numpy() if "topk_indices" in kw else None
+        want_ok = orc.validate_step_inputs(H, Z, y, m, b.V, idx)
+        assert (step.status() == B.NPD_OK) == want_ok
+        return step
+
+    b = fresh()
+    clean = status_of(b)
+    assert clean.status() == B.NPD_OK
+    plain = run_step(b)                               # same results with and without the checks
+    assert torch.equal(clean.kl, plain.kl) and torch.equal(clean.d_weight, plain.d_weight)
+    on = torch.nonzero(b.loss_mask).flatten()
+    off = torch.nonzero(b.loss_mask == 0).flatten()
+
+    b = fresh(); b.labels[int(on[3])] = b.V           # a label that names no class
+    assert status_of(b).status() == B.NPD_EDATA
+    b = fresh(); b.teacher[int(on[5]), :] = float("-inf")
+    assert status_of(b).status() == B.NPD_EDATA       # a loss token without any support
+    b = fresh(); b.teacher[int(on[5]), 1:] = float("-inf")
+    assert status_of(b).status() == B.NPD_OK          # one class left
+    b = fresh(); b.teacher[int(off[0]), :] = float("nan"); b.hidden[int(off[0]), :] = float("inf")
+    assert status_of(b).status() == B.NPD_OK          # rows of tokens without loss are not read
+    b = fresh(); b.teacher[int(on[-1]), b.V - 1] = float("nan")
+    assert status_of(b).status() == B.NPD_EDATA
+    b = fresh(); b.hidden[int(on[0]), 7] = float("inf")
+    assert status_of(b).status() == B.NPD_EDATA
+    # top-k teacher: stored indices must lie inside the vocabulary
+    b = fresh()
+    vals, idx = b.teacher.float().topk(4, dim=1)
+    idx = idx.to(torch.int32).contiguous()
+    assert status_of(b, topk_values=vals.contiguous(), topk_indices=idx).status() == B.NPD_OK
+    idx2 = idx.clone(); idx2[int(on[2]), 1] = b.V
+    assert status_of(b, topk_values=vals.contiguous(), topk_indices=idx2).status() == B.NPD_EDATA
