@@ -23,10 +23,11 @@
 // Two CTAs on neighbouring SMs (a cluster of 2) work as a pair on a 256 x 512 output tile
 // with tcgen05 .cta_group::2 (two M=256, N=256 accumulators that share the A operand): per
 // k-step each CTA stages its own 128 rows of A and its own half (128 rows) of each of the two
-// 256-row blocks of B, 48 KB for 2 x 128 x 256 x 64 MACs per SM.  The kernels here are bound by
-// the L2-to-SM operand traffic, and this tile moves a quarter fewer bytes per MAC than a
-// 256 x 256 pair tile; the price is that the 512 accumulator columns fill tensor memory, so
-// the drain of a tile is not overlapped with the next tile's MMAs (a few per cent at the
+// 256-row blocks of B, 48 KB for 2 x 128 x 256 x 64 MACs per SM.  This tile moves a quarter
+// fewer operand bytes per MAC than a 256 x 256 pair tile (less power under the board's cap) and
+// issues eight MMAs per k-step instead of four, which spreads the fixed cost of a k-step over
+// twice the work; the price is that the 512 accumulator columns fill tensor memory, so the
+// drain of a tile is not overlapped with the next tile's MMAs (a few per cent at the
 // k-extents used here).
 //
 // One CTA per SM, 384 threads: warp 0 = TMA producer, warp 1 = TMEM owner and, in the leader

@@ -107,8 +107,8 @@ constexpr int ZSUB_BYTES = BM * ZSUB_COLS * 2;  // 16 KB
 constexpr int THREADS = 384;
 constexpr int TMEM_COLS = 512;
 // Shared-memory layout.  224 KB go to the operand ring (32 KB per stage) and to the teacher
-// stages (16 KB each, per column half).  Both kernels are bound by the operand feed from L2,
-// not by its latency, so ring depth beyond four buys nothing; the forward pass puts the spare
+// stages (16 KB each, per column half).  Four operand stages cover the latency of the loads
+// (measured: five or six give the same time, two cost 8 %); the forward pass puts the spare
 // 32 KB into a third teacher stage per half (measured: 1.3 % faster), the gradient pass, whose
 // teacher stages double as staging for the gradient tiles, is faster with 5 + 2.
 template <int kMode>
