@@ -24,12 +24,13 @@
 // the logits of its own 128 tokens for all 256 columns.
 //
 // CTA = 384 threads, one CTA per SM, persistent over work units:
-//   warp 0      TMA producer for this CTA's H and W operand stages (4- or 5-stage ring); the
+//   warp 0      TMA producer for this CTA's H and W operand stages (a ring of 3 stages of two k-steps in the
+//               forward pass, of 5 single k-steps in the gradient pass); the
 //               completion of both CTAs' loads is counted on the leader's "full" barrier
 //   warp 1      leader CTA (cluster rank 0) only: tcgen05.mma issuer for the pair; commits
 //               are multicast so that "stage free" and "accumulator ready" reach both CTAs.
 //               In both CTAs this warp owns the 512 TMEM columns (2 accumulators 128x256).
-//   warp 2      TMA producer for this CTA's teacher sub-tiles (a ring of 2 or 3 stages per column half); the rows of a
+//   warp 2      TMA producer for this CTA's teacher sub-tiles (a ring of 1 or 2 stages per column half); the rows of a
 //               block lie anywhere in the packed batch, so each lane gathers four of them
 //   warp 3      gradient pass only: one thread hands each finished gradient sub-tile to a TMA
 //               store and recycles the stage when the store has read it
@@ -106,18 +107,25 @@ constexpr int ZSUB_COLS = 64;              // teacher sub-tile: 128 rows x 64 bf
 constexpr int ZSUB_BYTES = BM * ZSUB_COLS * 2;  // 16 KB
 constexpr int THREADS = 384;
 constexpr int TMEM_COLS = 512;
-// Shared-memory layout.  224 KB go to the operand ring (32 KB per stage) and to the teacher
-// stages (16 KB each, per column half).  Four operand stages cover the latency of the loads
-// (measured: five or six give the same time, two cost 8 %); the forward pass puts the spare
-// 32 KB into a third teacher stage per half (measured: 1.3 % faster), the gradient pass, whose
-// teacher stages double as staging for the gradient tiles, is faster with 5 + 2.
+// Shared-memory layout: 224 KB for the operand ring and the teacher stages (16 KB each, per
+// column half).
+// Every hand-off of an operand stage (the MMA issuer's wait for its loads, the release back to the
+// TMA producer) costs the tensor pipe about 120 clocks whatever the stage holds, so the forward
+// pass makes a stage two k-steps deep (64 KB, eight MMAs per hand-off instead of four): measured
+// 10 % faster than single-k-step stages holding the same bytes.  Three such stages cover the latency
+// of the loads; the 32 KB that remain give one teacher stage per half, which the forward epilogue
+// tolerates (its warps hand a sub-tile back as soon as they have read it).  The gradient pass does
+// not: its teacher stages double as staging for the gradient sub-tiles and are handed back only
+// when the store of a sub-tile has read it, so it needs two of them per half and keeps five
+// single-k-step operand stages (every variant with 64 KB stages was 9-24 % slower there).
 template <int kMode>
 struct Layout {
-  static constexpr int STAGES = kMode == 0 ? 4 : 5;  // operand ring depth
-  static constexpr int ZQ = kMode == 0 ? 3 : 2;      // teacher ring depth per column half
+  static constexpr int KS = kMode == 0 ? 2 : 1;      // k-steps per operand stage
+  static constexpr int STAGES = kMode == 0 ? 3 : 5;  // operand ring depth
+  static constexpr int ZQ = kMode == 0 ? 1 : 2;      // teacher ring depth per column half
   static constexpr int OFF_A = 0;
-  static constexpr int OFF_B = OFF_A + STAGES * A_BYTES;
-  static constexpr int OFF_Z = OFF_B + STAGES * B_BYTES;
+  static constexpr int OFF_B = OFF_A + STAGES * KS * A_BYTES;
+  static constexpr int OFF_Z = OFF_B + STAGES * KS * B_BYTES;
   static constexpr int OFF_BAR = OFF_Z + 2 * ZQ * ZSUB_BYTES;
   static constexpr int NUM_BARS = 2 * STAGES + 4 + 6 * ZQ;
   static constexpr int SMEM_BYTES = OFF_BAR + NUM_BARS * 8 + 16 + 1024;
@@ -137,7 +145,7 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                const KdTileParams p) {
   using namespace kd_cfg;
   using L = Layout<kMode>;
-  constexpr int STAGES = L::STAGES, ZQ = L::ZQ, OFF_A = L::OFF_A, OFF_B = L::OFF_B, OFF_Z = L::OFF_Z,
+  constexpr int KS = L::KS, STAGES = L::STAGES, ZQ = L::ZQ, OFF_A = L::OFF_A, OFF_B = L::OFF_B, OFF_Z = L::OFF_Z,
                 OFF_BAR = L::OFF_BAR, NUM_BARS = L::NUM_BARS;
   constexpr int ZC = kTeacherF32 ? 32 : ZSUB_COLS;  // columns of a teacher sub-tile (128-byte rows)
   extern __shared__ uint8_t smem_raw[];
@@ -224,15 +232,18 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
         run_of(u, slot, r, s, vt0, vt1);
         const int rl = r < 0 ? 0 : r;
         for (int vt = vt0; vt < vt1 && ok; ++vt) {
-          for (int ks = 0; ks < p.ksteps; ++ks, ++it) {
+          for (int ks = 0; ks < p.ksteps; ks += KS, ++it) {
             const uint32_t st = it % STAGES, ph = (it / STAGES) & 1;
+            const int nk = min(KS, p.ksteps - ks);  // k-steps this stage carries
             if (!(ok = mbar_wait(empty0 + 8 * st, ph ^ 1, abort_flag))) break;
             // the leader's barrier counts the bytes of both CTAs' loads of this stage
-            if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, 2 * (A_BYTES + B_BYTES));
+            if (rank == 0) mbar_arrive_expect_tx(full0 + 8 * st, 2 * nk * (A_BYTES + B_BYTES));
             const uint32_t fb = full_leader + 8 * st;
-            tma_load_2d_pair(smem_u32(smem + OFF_A + st * A_BYTES), &tmap_h, fb, ks * BK, rl);
-            tma_load_2d_pair(smem_u32(smem + OFF_B + st * B_BYTES), &tmap_w, fb, ks * BK,
-                             vt * BN + static_cast<int>(rank) * BNH);
+            for (int h = 0; h < nk; ++h) {
+              tma_load_2d_pair(smem_u32(smem + OFF_A + (st * KS + h) * A_BYTES), &tmap_h, fb, (ks + h) * BK, rl);
+              tma_load_2d_pair(smem_u32(smem + OFF_B + (st * KS + h) * B_BYTES), &tmap_w, fb, (ks + h) * BK,
+                               vt * BN + static_cast<int>(rank) * BNH);
+            }
           }
         }
       }
@@ -272,17 +283,20 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
           if (!(ok = mbar_wait(tempty0 + 8 * buf, tph ^ 1, abort_flag))) break;
           tc_fence_after_sync();
           const uint32_t d_tmem = tmem_base + buf * BN;
-          for (int ks = 0; ks < p.ksteps; ++ks, ++it) {
+          for (int ks = 0; ks < p.ksteps; ks += KS, ++it) {
             const uint32_t st = it % STAGES, ph = (it / STAGES) & 1;
+            const int nk = min(KS, p.ksteps - ks);
             if (!(ok = mbar_wait(full0 + 8 * st, ph, abort_flag))) break;
             tc_fence_after_sync();
-            const uint32_t sa = smem_u32(smem + OFF_A + st * A_BYTES);
-            const uint32_t sb = smem_u32(smem + OFF_B + st * B_BYTES);
+            for (int h = 0; h < nk; ++h) {
+              const uint32_t sa = smem_u32(smem + OFF_A + (st * KS + h) * A_BYTES);
+              const uint32_t sb = smem_u32(smem + OFF_B + (st * KS + h) * B_BYTES);
 #pragma unroll
-            for (int k = 0; k < BK / UK; ++k) {
-              umma_bf16_pair(d_tmem, umma_desc_sw128(sa + k * (UK * 2), 16, 1024),
-                             umma_desc_sw128(sb + k * (UK * 2), 16, 1024), idesc,
-                             (ks > 0 || k > 0) ? 1u : 0u);
+              for (int k = 0; k < BK / UK; ++k) {
+                umma_bf16_pair(d_tmem, umma_desc_sw128(sa + k * (UK * 2), 16, 1024),
+                               umma_desc_sw128(sb + k * (UK * 2), 16, 1024), idesc,
+                               (ks > 0 || h > 0 || k > 0) ? 1u : 0u);
+              }
             }
             umma_commit_pair(empty0 + 8 * st);
           }
