@@ -468,11 +468,12 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                 const uint32_t w[4] = {zq[i].x, zq[i].y, zq[i].z, zq[i].w};
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
+                  // (the gradient pass needs no clamp: 2^(-inf) is an exact zero there)
                   if (kTeacherF32) {
-                    zt[4 * i + k] = fmaxf(__uint_as_float(w[k]), kNegClamp);
+                    zt[4 * i + k] = kMode == kForward ? fmaxf(__uint_as_float(w[k]), kNegClamp) : __uint_as_float(w[k]);
                   } else {
-                    zt[8 * i + 2 * k] = fmaxf(bf16_lo(w[k]), kNegClamp);
-                    zt[8 * i + 2 * k + 1] = fmaxf(bf16_hi(w[k]), kNegClamp);
+                    zt[8 * i + 2 * k] = kMode == kForward ? fmaxf(bf16_lo(w[k]), kNegClamp) : bf16_lo(w[k]);
+                    zt[8 * i + 2 * k + 1] = kMode == kForward ? fmaxf(bf16_hi(w[k]), kNegClamp) : bf16_hi(w[k]);
                   }
                 }
               }
@@ -570,9 +571,14 @@ kd_tile_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid_constant
                   }
                 }
               }
+              if (nvalid >= 32) {
 #pragma unroll
-              for (int i = 0; i < 32; i += 2)
-                packed[i >> 1] = pack_bf16x2(i < nvalid ? g[i] : 0.f, i + 1 < nvalid ? g[i + 1] : 0.f);
+                for (int i = 0; i < 32; i += 2) packed[i >> 1] = pack_bf16x2(g[i], g[i + 1]);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2)
+                  packed[i >> 1] = pack_bf16x2(i < nvalid ? g[i] : 0.f, i + 1 < nvalid ? g[i + 1] : 0.f);
+              }
               if (kTeacherF32) {
                 // 64-byte gradient rows, dense from the start of the stage: they overlap other
                 // threads' teacher rows, so everyone of this half must have read its row first
